@@ -1,0 +1,411 @@
+"""Benchmark: IST training samples/s on one B200 (or N independent replicas).
+
+A "step" is one whole IST round on a synthetic workload: partition + gather, K local SGD steps
+of all S subnets, reassemble.  Timed on the device with CUDA events on the library's stream,
+after warm-up, bracketed by a barrier and a synchronize; max over ranks.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C3] [--impl reference]
+
+Prints one JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1910_02120_b200 import synth  # noqa: E402
+
+METRIC = "IST training samples/sec (all S subnets, device-timed)"
+UNIT = "samples/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="C3", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+def config_dict(w: synth.Workload, n_gpus: int):
+    return {
+        "workload": f"{w.name}: MLP {'-'.join(map(str, w.layer_dims))}, S={w.S}, batch={w.B}, "
+                    f"K={w.K} local steps/round, {w.precision} operands, fp32 masters",
+        "samples_per_step": w.samples_per_round,
+        "step": "one IST round: partition+gather, K local SGD steps of S subnets, reassemble",
+        "inputs": f"{w.x_dist}; distinct batch per subnet per local step",
+        "l2": "per-round working set (inputs + full network + packed slices) exceeds the 126 MB L2",
+        "parallelism": "single GPU" if n_gpus == 1 else f"{n_gpus} independent replicas",
+    }
+
+
+# ---------------------------------------------------------------------------------------------
+# algorithmic work per round (all S subnets), used for the roofline fractions
+# ---------------------------------------------------------------------------------------------
+
+def work_model(w: synth.Workload):
+    d, S, B, K = w.layer_dims, w.S, w.B, w.K
+    t = len(d) - 1
+    n = [d[0]] + [-(-d[l] // S) for l in range(1, t)] + [d[t]]
+    layer_elems = [n[l - 1] * n[l] for l in range(1, t + 1)]          # per subnet
+    packed = S * sum(layer_elems)
+    dense_first = w.x_dist != "csr"
+    fwd = 2 * B * S * sum(layer_elems[(0 if dense_first else 1):])
+    dx = 2 * B * S * sum(layer_elems[1:])
+    dw = 2 * B * S * sum(layer_elems[(0 if dense_first else 1):])
+    opw = 2 if w.precision == "bf16" else 0
+    return {
+        "packed_elems": packed,
+        "flops": {"fwd": fwd * K, "dx": dx * K, "dw_sgd": dw * K},
+        # bytes: gather = read fp32 + write fp32 master (+ bf16 copy); scatter = read + write fp32;
+        # fused update inside dw_sgd = read + write master (+ bf16 copy)
+        "bytes": {"gather": packed * (8 + opw), "scatter": packed * 8,
+                  "dw_sgd": packed * (8 + opw) * K},
+    }
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1]))
+                mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[5:9]):
+                if v.strip().lower() == "active":
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ---------------------------------------------------------------------------------------------
+# the CPU oracle, timed as it stands on a bounded sample of the workload
+# ---------------------------------------------------------------------------------------------
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+class OracleSample:
+    """One bounded sample of a round: the full partition, the slicing of all S subnets, one local
+    step on each of `n_sub` subnets, and the reassembly.  The round's throughput is extrapolated
+    as S*K*B / (t_partition+slice+reassemble + S*K*t_step)."""
+
+    def __init__(self, w: synth.Workload, n_sub=1):
+        from oracle import ist_oracle as O
+        self.O, self.w, self.n_sub = O, w, min(n_sub, w.S)
+        W, b = synth.make_weights(w.layer_dims, w.seed)
+        self.o = O.IstOracle(w.layer_dims, w.S)
+        self.o.bind_weights(W, b)
+        del W, b
+        small = w.scaled(S=self.n_sub, K=1)
+        self.data = synth.make_round_inputs(small)
+
+    def run(self, seed):
+        o, w = self.o, self.w
+        t0 = time.perf_counter()
+        o.partition(seed)
+        t1 = time.perf_counter()
+        X = (self.data.row_ptr, self.data.col, self.data.val) if self.data.is_csr else self.data.X
+        for s in range(self.n_sub):
+            Ws, bs = o.subnets[s]
+            xb, yb = o._batch(X, self.data.y, s, 0)
+            self.O.sgd_step(Ws, bs, xb, yb, w.lr, o.dtype)
+        t2 = time.perf_counter()
+        o.reassemble()
+        t3 = time.perf_counter()
+        fixed = (t1 - t0) + (t3 - t2)
+        step = (t2 - t1) / self.n_sub
+        est_round = fixed + w.S * w.K * step
+        return w.samples_per_round / est_round, t3 - t0
+
+    def describe(self):
+        return (f"per step: partition + slicing of all {self.w.S} subnets + 1 local SGD step on "
+                f"{self.n_sub} subnet(s) at full width + reassembly, fp64 numpy; round throughput "
+                f"extrapolated as S*K*B/(t_fixed + S*K*t_step)")
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    smp = OracleSample(w)
+    for i in range(args.warmup):
+        smp.run(1000 + i)
+    vals, secs = [], []
+    for i in range(args.steps):
+        v, s = smp.run(2000 + i)
+        vals.append(v)
+        secs.append(s)
+    value = float(np.mean(vals))
+    cores = oracle_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(secs)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": config_dict(w, 1),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": smp.describe()},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# the CUDA path
+# ---------------------------------------------------------------------------------------------
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_1910_02120_b200 import api
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- inputs, resident on the device before timing starts ---------------------------------
+    ww = w.scaled(seed=w.seed + 1000 * rank)
+    W, b = synth.make_weights(ww.layer_dims, ww.seed)
+    Wd = [torch.from_numpy(x).to(dev) for x in W]
+    bd = [torch.from_numpy(x).to(dev) for x in b]
+    del W, b
+    data = synth.make_round_inputs(ww)
+    prec = api.IST_BF16 if w.precision == "bf16" else api.IST_FP32
+    ctx = api.Ist(w.layer_dims, w.S, prec, w.B, input_is_csr=data.is_csr, device=str(dev))
+    ctx.bind_weights(Wd, bd)
+    y_host = torch.from_numpy(data.y.reshape(-1).copy()).pin_memory()
+    if data.is_csr:
+        host_in = [torch.from_numpy(data.row_ptr.astype(np.int32)).pin_memory(),
+                   torch.from_numpy(data.col).pin_memory(), torch.from_numpy(data.val).pin_memory()]
+    else:
+        xt = torch.from_numpy(data.X.reshape(-1, w.layer_dims[0]))
+        if w.precision == "bf16" and w.layer_dims[0] % 8 == 0:
+            xt = xt.to(torch.bfloat16)
+        host_in = [xt.pin_memory()]
+    dev_in = [t.to(dev) for t in host_in]
+    y_dev = y_host.to(dev)
+    loss_dev = torch.empty(w.S * w.K, dtype=torch.float32, device=dev)
+    loss_host = torch.empty(w.S * w.K, dtype=torch.float32).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host_in) + y_host.numel() * 4
+    d2h = loss_host.numel() * 4
+
+    def X_of(ts):
+        return tuple(ts) if data.is_csr else ts[0]
+
+    def one_round(r, X, y):
+        ctx.round(7000 + r, X, y, w.lr, w.K, w.B, loss_out=loss_dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def max_over_ranks(ms):
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return ms
+
+    # ---- device-resident timing ---------------------------------------------------------------
+    for i in range(max(args.warmup, 3)):
+        one_round(i, X_of(dev_in), y_dev)
+    ctx.sync_status()
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    launches0 = ctx.kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        one_round(100 + i, X_of(dev_in), y_dev)
+    e1.record()
+    barrier()
+    launches = ctx.kernel_launches() - launches0
+    clocks = sampler.stop()
+    ms = max_over_ranks(e0.elapsed_time(e1))
+    ctx.sync_status()
+    value = world * w.samples_per_round * args.steps / (ms * 1e-3)
+
+    # ---- end to end: host buffers in, loss out, copies inside the timed region ------------------
+    stage_in = [torch.empty_like(t, device=dev) for t in host_in]
+    stage_y = torch.empty_like(y_host, device=dev)
+
+    def e2e_round(r):
+        for dst, src in zip(stage_in, host_in):
+            dst.copy_(src, non_blocking=True)
+        stage_y.copy_(y_host, non_blocking=True)
+        one_round(r, X_of(stage_in), stage_y)
+        loss_host.copy_(loss_dev, non_blocking=True)
+
+    e2e_round(0)
+    barrier()
+    e0.record()
+    for i in range(args.steps):
+        e2e_round(200 + i)
+    e1.record()
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1))
+    e2e_value = world * w.samples_per_round * args.steps / (ms_e2e * 1e-3)
+
+    # ---- per-kernel-class device times (separate pass, events around each class) ---------------
+    ctx.profile(True)
+    prof_rounds = min(args.steps, 3)
+    for i in range(prof_rounds):
+        one_round(300 + i, X_of(dev_in), y_dev)
+    prof = ctx.profile_read()
+    ctx.profile(False)
+    ctx.sync_status()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    wm = work_model(w)
+    tensor_peak = pk["bf16_tflops_sustained"] if w.precision == "bf16" else None
+    kernels = {}
+    for name, (n, t_ms) in prof.items():
+        if n == 0:
+            continue
+        ent = {"launches_per_step": n / prof_rounds, "ms_per_step": t_ms / prof_rounds}
+        sec = t_ms * 1e-3 / prof_rounds
+        if name in wm["flops"] and sec > 0:
+            ent["tflops"] = wm["flops"][name] / sec / 1e12
+        if name in wm["bytes"] and sec > 0:
+            ent["gbs"] = wm["bytes"][name] / sec / 1e9
+        kernels[name] = ent
+    dominant = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    dk = kernels[dominant]
+    if dominant in wm["flops"] and tensor_peak:
+        per_launch = wm["flops"][dominant] / dk["launches_per_step"]
+        achieved = dk["tflops"]
+        roof = {"kernel": dominant, "bound": "tensor", "achieved": achieved, "peak": tensor_peak,
+                "unit": "TFLOP/s", "frac": achieved / tensor_peak, "traffic": None,
+                "peak_source": pk["_source"] + " (sustained bf16)", "flops_per_launch": per_launch,
+                "avg_launch_ms": dk["ms_per_step"] / dk["launches_per_step"]}
+    elif dominant in wm["flops"]:
+        # fp32 CUDA-core contraction: 148 SMs x 128 FMA lanes x 2 flop x max clock
+        alu_peak = 148 * 128 * 2 * pk.get("sm_max_mhz", 1965.0) * 1e6 / 1e12
+        roof = {"kernel": dominant, "bound": "alu", "achieved": dk["tflops"], "peak": alu_peak,
+                "unit": "TFLOP/s", "frac": dk["tflops"] / alu_peak, "traffic": None,
+                "peak_source": "derived: 148 SMs x 128 lanes x 2 x max SM clock"}
+    else:
+        gbs = dk.get("gbs", 0.0)
+        roof = {"kernel": dominant, "bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / pk["hbm_gbs"], "traffic": None, "peak_source": pk["_source"]}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        smp = OracleSample(w, n_sub=2)
+        t0 = time.perf_counter()
+        vals = []
+        while len(vals) < 2 or (time.perf_counter() - t0 < 10 and len(vals) < 6):
+            vals.append(smp.run(9000 + len(vals))[0])
+        cpu = {"value": float(np.mean(vals)), "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+               "sample": smp.describe() + f"; {len(vals)} samples"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": w.precision.replace("fp", "f"), "data": "synthetic",
+        "config": config_dict(w, world), "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": launches, "roofline": roof, "kernels": kernels, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    w = synth.WORKLOADS[args.config]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,204 @@
+/*
+ * libist — one round of Independent Subnet Training (IST, arXiv 1910.02120) on one GPU.
+ *
+ * A round (Sec. 2.1 "Methodology" of the paper): the hidden neurons of a fully connected
+ * network are randomly partitioned into S disjoint groups ("Constructing Subnets"), every
+ * subnet takes the weight slices its neurons select, trains for K iterations of local SGD
+ * without talking to the others ("Training Subnets"; K is the paper's J), and the slices are
+ * copied back into the full network.  The paper places the S subnets on S machines; here they
+ * are S groups of one grouped computation on a single device.
+ *
+ * Conventions
+ *   - C ABI, no exceptions.  Every call returns ist_status (0 = IST_OK, < 0 = error) unless
+ *     stated otherwise; ist_last_error() gives a human-readable message for the last failure.
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host memory.
+ *   - The library allocates no device memory.  The caller owns the full network, the inputs,
+ *     the outputs and one workspace blob (size from ist_workspace_bytes) that must stay alive
+ *     and untouched from ist_create to ist_destroy.
+ *   - All device work is enqueued on the stream given to ist_create, in call order, and is
+ *     asynchronous to the host.  Only ist_sync_status() synchronises.
+ *   - Network layout: layer_dims = {N_0, ..., N_t}; layer l (1..t) has W_l row-major
+ *     [N_{l-1}][N_l] fp32 (y = x * W_l + b_l) and b_l [N_l] fp32.  Hidden layers use ReLU;
+ *     the loss is the softmax cross-entropy averaged over the minibatch.  (The paper fixes
+ *     neither the loss nor biases; these are this library's reading.)
+ *   - Call order: ist_create -> ist_bind_weights -> { ist_partition -> ist_local_steps* ->
+ *     ist_reassemble }* ; ist_eval any time the network is bound and not partitioned.
+ *     Between ist_partition and ist_reassemble the caller must not write the bound weights.
+ */
+#ifndef IST_H_
+#define IST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ist_ctx ist_ctx; /* opaque, host object */
+typedef int32_t ist_status;
+
+enum {
+  IST_OK = 0,
+  IST_ERR_ARG = -1,            /* null pointer, size out of range, misaligned pointer */
+  IST_ERR_STATE = -2,          /* call out of order */
+  IST_ERR_WORKSPACE = -3,      /* workspace too small or misaligned */
+  IST_ERR_CUDA = -4,           /* a CUDA runtime call failed */
+  IST_ERR_DEVICE_CHECK = -5,   /* a device-side bounds check tripped (label / column / index) */
+  IST_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait gave up */
+  IST_ERR_UNSUPPORTED = -7     /* valid request this build cannot serve */
+};
+
+/* Operand precision of the local steps.  Master weights are fp32 in both modes. */
+enum { IST_FP32 = 0, IST_BF16 = 1 };
+
+/* Input kinds. */
+enum { IST_X_DENSE_F32 = 0, IST_X_DENSE_BF16 = 1, IST_X_CSR = 2 };
+
+/*
+ * Minibatches for ist_local_steps / ist_eval.  X is logically [S][K][batch][N_0]: subnet s at
+ * local step k reads rows  r0 = s*stride_subnet + k*stride_step ... r0 + batch - 1  (strides in
+ * rows; 0 means "the same rows again").  The paper gives every site its own data and draws a
+ * minibatch per iteration (Sec. 2.1); the two strides express that.
+ *   dense : `dense` points at row-major rows of N_0 elements (fp32 or bf16), device memory.
+ *           bf16 rows need N_0 % 8 == 0 and a 16-byte aligned base.
+ *   CSR   : row_ptr [rows+1] (absolute offsets into col/val), col [nnz] (0 <= col < N_0,
+ *           distinct inside a row), val [nnz] fp32; all device memory.
+ * ist_eval ignores the strides and reads rows 0..n-1.
+ */
+typedef struct ist_input {
+  int32_t kind;
+  int32_t batch;
+  const void* dense;
+  const int32_t* row_ptr;
+  const int32_t* col;
+  const float* val;
+  int64_t stride_subnet;
+  int64_t stride_step;
+} ist_input;
+
+/*
+ * Bytes of device workspace a context of this shape needs (0 on invalid arguments).
+ * layer_dims: host, n_dims = t+1 entries, each >= 1.  S >= 1 subnets (S = 1 if t = 1),
+ * S <= every hidden N_l.  max_batch >= 1: largest `batch` later passed in ist_input
+ * (ist_eval processes its rows in chunks of max_batch).
+ */
+size_t ist_workspace_bytes(const int64_t* layer_dims, int n_dims, int S, int precision,
+                           int max_batch, int input_is_csr);
+
+/*
+ * Creates a context.  workspace_dev: device, 256-byte aligned, >= ist_workspace_bytes(...).
+ * cuda_stream: a cudaStream_t (NULL = legacy default stream), borrowed.  The workspace is
+ * cleared on this stream.  *out is set only on success; free it with ist_destroy.
+ */
+ist_status ist_create(ist_ctx** out, const int64_t* layer_dims, int n_dims, int S, int precision,
+                      int max_batch, int input_is_csr, void* workspace_dev, size_t workspace_bytes,
+                      void* cuda_stream);
+
+/*
+ * The full network the rounds act on.  W_dev / b_dev: host arrays of t device pointers
+ * (W_l [N_{l-1}][N_l] fp32, b_l [N_l] fp32), borrowed until ist_destroy or the next bind.
+ */
+ist_status ist_bind_weights(ist_ctx* ctx, float* const* W_dev, float* const* b_dev);
+
+/*
+ * Sec. 2.1 "Constructing Subnets" + distribution of the slices.  Draws a fresh partition of
+ * every hidden layer from `seed` and gathers each subnet's slices into the workspace:
+ * subnet s owns W_1[:, G_1^s], W_l[G_{l-1}^s, G_l^s] for 1 < l < t, W_t[G_{t-1}^s, :], the
+ * hidden biases of its neurons and its own copy of the output bias (App. A: each neuron in
+ * exactly one subnet; footnote: inactive neurons are never computed).
+ * Partition rule (the paper states only "uniform assignment"): neuron i of hidden layer l
+ * gets the i-th output of a SplitMix64 generator seeded with the l-th output of a SplitMix64
+ * generator seeded with `seed`; neurons are ranked by (key, index); group g takes the next
+ * floor(N_l/S) (+1 if g < N_l mod S) ranks; indices are ascending inside a group.
+ */
+ist_status ist_partition(ist_ctx* ctx, uint64_t seed);
+
+/*
+ * Copies the current partition of hidden layer `hidden_layer` (1..t-1) out:
+ * idx_out_dev [N_l] int32 (group-major, ascending inside a group), off_out_dev [S+1] int32.
+ */
+ist_status ist_get_partition(ist_ctx* ctx, int hidden_layer, int32_t* idx_out_dev,
+                             int32_t* off_out_dev);
+
+/*
+ * Copies subnet s's current fp32 master slice of layer l (1..t) out, densely:
+ * W_out_dev [rows][cols] with rows = |G_{l-1}^s| (N_0 for l = 1), cols = |G_l^s| (N_t for
+ * l = t); b_out_dev [cols].  Either pointer may be NULL.  Needs a partition in place.
+ */
+ist_status ist_get_subnet_params(ist_ctx* ctx, int layer, int s, float* W_out_dev,
+                                 float* b_out_dev);
+
+/*
+ * Sec. 2.1 "Training Subnets": K iterations of local SGD on every subnet, no exchange.
+ * Step k of subnet s: forward (App. A Eq. (2) on the slice, without the n^2 factor, as
+ * Sec. 2.2 removes it), mean softmax cross-entropy against y, backward, w <- w - lr * grad
+ * with all gradients taken at the pre-update weights.
+ * y_dev: int32 labels addressed like X rows (row r -> y_dev[r]), 0 <= y < N_t.
+ * loss_out_dev: [S*K] fp32, loss_out[s*K + k] = loss of subnet s before the update of step k
+ * (may be NULL).  1 <= K.  X->batch <= max_batch.
+ */
+ist_status ist_local_steps(ist_ctx* ctx, const ist_input* X, const int32_t* y_dev, float lr, int K,
+                           float* loss_out_dev);
+
+/*
+ * Sec. 2.1: "subnet parameters are copied back into the full NN, where no collisions occur".
+ * Writes every trained slice to the positions it was gathered from; entries of middle layers
+ * whose row group differs from their column group are not written.  The output bias, the one
+ * parameter all subnets hold, becomes b + (sum_s (b^(s) - b)) / S (its mean over the copies).
+ * Afterwards the context is back in the "bound" state.
+ */
+ist_status ist_reassemble(ist_ctx* ctx);
+
+/*
+ * Full-width forward pass of the bound network (the deployed model, Sec. 2.2) over n rows:
+ * mean softmax cross-entropy -> *mean_loss_out_dev (fp32), number of rows whose arg-max
+ * (lowest index on ties) equals the label -> *n_correct_out_dev (int64).  Computed in fp32.
+ */
+ist_status ist_eval(ist_ctx* ctx, const ist_input* X, const int32_t* y_dev, int64_t n,
+                    float* mean_loss_out_dev, int64_t* n_correct_out_dev);
+
+/* Waits for the stream and returns the sticky device status (IST_OK, IST_ERR_DEVICE_CHECK,
+ * IST_ERR_DEVICE_TIMEOUT or IST_ERR_CUDA). */
+ist_status ist_sync_status(ist_ctx* ctx);
+
+/*
+ * Measurement aid (no counterpart in the paper).  Kernel classes of a round, in the order a
+ * round runs them.  With profiling enabled every group of launches of one class is bracketed
+ * by a pair of CUDA events on the context's stream; ist_profile_read synchronises and returns
+ * the number of kernels launched and the summed device time of that class since profiling was
+ * enabled.  Enabling clears earlier records.  The events cost a few microseconds each, so
+ * throughput should be timed with profiling off.
+ */
+enum {
+  IST_K_PARTITION = 0, /* keys, ranks, index lists */
+  IST_K_GATHER = 1,    /* full network -> packed slices (+ bf16 copies) */
+  IST_K_STAGE = 2,     /* fp32 input rows -> bf16 staging */
+  IST_K_FWD = 3,       /* forward GEMMs with bias / ReLU / logits epilogues */
+  IST_K_LOSS = 4,      /* softmax cross-entropy, loss reduction */
+  IST_K_DX = 5,        /* delta_{l-1} GEMMs with the ReLU mask epilogue */
+  IST_K_DW_SGD = 6,    /* weight-gradient GEMMs with the fused SGD update */
+  IST_K_BIAS_SGD = 7,  /* bias gradient and update */
+  IST_K_SPMM = 8,      /* sparse first layer: forward, backward + update */
+  IST_K_SCATTER = 9,   /* packed slices -> full network */
+  IST_K_EVAL = 10,     /* full-width evaluation */
+  IST_K_COUNT = 11
+};
+ist_status ist_profile(ist_ctx* ctx, int enable);
+ist_status ist_profile_read(ist_ctx* ctx, int kernel_class, int64_t* launches_out_host,
+                            double* ms_out_host);
+
+/* Number of kernels this context has launched so far (host counter). */
+int64_t ist_kernel_launches(const ist_ctx* ctx);
+
+/* Message for the most recent failing call on this context ("" if none).  ctx may be NULL,
+ * in which case the message of the last failing ist_create on this thread is returned. */
+const char* ist_last_error(const ist_ctx* ctx);
+
+/* Frees the host object.  Does not touch device memory; pending work keeps running. */
+void ist_destroy(ist_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IST_H_ */

@@ -1,0 +1,267 @@
+"""ctypes binding of libist.so: the same calls as include/ist.h, with torch tensors as the
+owners of device memory.  Argument marshalling only; every step of a round runs inside the
+library's CUDA kernels.  There is no CPU fallback: if the shared library is missing, import
+fails with instructions to build it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libist.so")
+
+IST_OK = 0
+IST_ERR_ARG, IST_ERR_STATE, IST_ERR_WORKSPACE, IST_ERR_CUDA = -1, -2, -3, -4
+IST_ERR_DEVICE_CHECK, IST_ERR_DEVICE_TIMEOUT, IST_ERR_UNSUPPORTED = -5, -6, -7
+IST_FP32, IST_BF16 = 0, 1
+IST_X_DENSE_F32, IST_X_DENSE_BF16, IST_X_CSR = 0, 1, 2
+
+EXPORTS = [
+    "ist_workspace_bytes", "ist_create", "ist_bind_weights", "ist_partition", "ist_get_partition",
+    "ist_get_subnet_params", "ist_local_steps", "ist_reassemble", "ist_eval", "ist_sync_status",
+    "ist_kernel_launches", "ist_last_error", "ist_destroy", "ist_profile", "ist_profile_read",
+]
+
+KERNEL_CLASSES = ["partition", "gather", "stage", "fwd", "loss", "dx", "dw_sgd", "bias_sgd", "spmm",
+                  "scatter", "eval"]
+
+
+class IstInput(ctypes.Structure):
+    _fields_ = [
+        ("kind", ctypes.c_int32),
+        ("batch", ctypes.c_int32),
+        ("dense", ctypes.c_void_p),
+        ("row_ptr", ctypes.c_void_p),
+        ("col", ctypes.c_void_p),
+        ("val", ctypes.c_void_p),
+        ("stride_subnet", ctypes.c_int64),
+        ("stride_step", ctypes.c_int64),
+    ]
+
+
+class IstError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"ist_status {status}: {message}")
+        self.status = status
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_1910_02120_b200.build` "
+            "(needs nvcc); there is no fallback implementation")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, u64, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.c_size_t
+    p64 = ctypes.POINTER(ctypes.c_int64)
+    lib.ist_workspace_bytes.restype = sz
+    lib.ist_workspace_bytes.argtypes = [p64, i32, i32, i32, i32, i32]
+    lib.ist_create.restype = ctypes.c_int32
+    lib.ist_create.argtypes = [ctypes.POINTER(vp), p64, i32, i32, i32, i32, i32, vp, sz, vp]
+    lib.ist_bind_weights.restype = ctypes.c_int32
+    lib.ist_bind_weights.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
+    lib.ist_partition.restype = ctypes.c_int32
+    lib.ist_partition.argtypes = [vp, u64]
+    lib.ist_get_partition.restype = ctypes.c_int32
+    lib.ist_get_partition.argtypes = [vp, i32, vp, vp]
+    lib.ist_get_subnet_params.restype = ctypes.c_int32
+    lib.ist_get_subnet_params.argtypes = [vp, i32, i32, vp, vp]
+    lib.ist_local_steps.restype = ctypes.c_int32
+    lib.ist_local_steps.argtypes = [vp, ctypes.POINTER(IstInput), vp, ctypes.c_float, i32, vp]
+    lib.ist_reassemble.restype = ctypes.c_int32
+    lib.ist_reassemble.argtypes = [vp]
+    lib.ist_eval.restype = ctypes.c_int32
+    lib.ist_eval.argtypes = [vp, ctypes.POINTER(IstInput), vp, i64, vp, vp]
+    lib.ist_sync_status.restype = ctypes.c_int32
+    lib.ist_sync_status.argtypes = [vp]
+    lib.ist_kernel_launches.restype = i64
+    lib.ist_kernel_launches.argtypes = [vp]
+    lib.ist_last_error.restype = ctypes.c_char_p
+    lib.ist_last_error.argtypes = [vp]
+    lib.ist_profile.restype = ctypes.c_int32
+    lib.ist_profile.argtypes = [vp, i32]
+    lib.ist_profile_read.restype = ctypes.c_int32
+    lib.ist_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double)]
+    lib.ist_destroy.restype = None
+    lib.ist_destroy.argtypes = [vp]
+    return lib
+
+
+lib = _load()
+
+
+def _dims(layer_dims: Sequence[int]):
+    arr = (ctypes.c_int64 * len(layer_dims))(*[int(d) for d in layer_dims])
+    return arr, len(layer_dims)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _check(handle, status: int):
+    if status != IST_OK:
+        raise IstError(status, lib.ist_last_error(handle).decode())
+
+
+def ist_workspace_bytes(layer_dims, S, precision, max_batch, input_is_csr=False) -> int:
+    arr, n = _dims(layer_dims)
+    return int(lib.ist_workspace_bytes(arr, n, S, precision, max_batch, int(bool(input_is_csr))))
+
+
+def make_input(X, batch: int, stride_subnet: int, stride_step: int) -> Tuple[IstInput, tuple]:
+    """X: a CUDA tensor of rows (fp32 or bf16, last dim N_0) or a (row_ptr, col, val) triple of
+    CUDA tensors (int32, int32, fp32).  Returns the struct and the tensors it points into."""
+    inp = IstInput()
+    inp.batch = int(batch)
+    inp.stride_subnet = int(stride_subnet)
+    inp.stride_step = int(stride_step)
+    if isinstance(X, (tuple, list)):
+        rp, col, val = X
+        assert rp.dtype == torch.int32 and col.dtype == torch.int32 and val.dtype == torch.float32
+        assert rp.is_cuda and col.is_cuda and val.is_cuda
+        inp.kind = IST_X_CSR
+        inp.row_ptr, inp.col, inp.val = rp.data_ptr(), col.data_ptr(), val.data_ptr()
+        return inp, (rp, col, val)
+    assert X.is_cuda and X.is_contiguous()
+    if X.dtype == torch.float32:
+        inp.kind = IST_X_DENSE_F32
+    elif X.dtype == torch.bfloat16:
+        inp.kind = IST_X_DENSE_BF16
+    else:
+        raise TypeError(f"unsupported input dtype {X.dtype}")
+    inp.dense = X.data_ptr()
+    return inp, (X,)
+
+
+class Ist:
+    """One IST context: owns the workspace tensor, borrows the full network's tensors.
+
+    Method names mirror the C calls (ist_partition -> partition, ...)."""
+
+    def __init__(self, layer_dims: Sequence[int], S: int, precision: int, max_batch: int,
+                 input_is_csr: bool = False, device: str = "cuda:0", stream: Optional[torch.cuda.Stream] = None):
+        self.layer_dims = [int(d) for d in layer_dims]
+        self.t = len(self.layer_dims) - 1
+        self.S, self.precision, self.max_batch = int(S), int(precision), int(max_batch)
+        self.input_is_csr = bool(input_is_csr)
+        self.device = torch.device(device)
+        self.stream = stream
+        self.handle = ctypes.c_void_p()
+        nbytes = ist_workspace_bytes(self.layer_dims, S, precision, max_batch, input_is_csr)
+        if nbytes == 0:
+            raise IstError(IST_ERR_ARG, lib.ist_last_error(None).decode())
+        self.workspace_bytes = nbytes
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            arr, n = _dims(self.layer_dims)
+            st = lib.ist_create(ctypes.byref(self.handle), arr, n, self.S, self.precision, self.max_batch,
+                                int(self.input_is_csr), self.workspace.data_ptr(), nbytes, self._stream_ptr())
+        if st != IST_OK:
+            self.handle = ctypes.c_void_p()
+            raise IstError(st, lib.ist_last_error(None).decode())
+        self.W: List[torch.Tensor] = []
+        self.b: List[torch.Tensor] = []
+
+    def _stream_ptr(self):
+        s = self.stream if self.stream is not None else torch.cuda.current_stream(self.device)
+        return ctypes.c_void_p(s.cuda_stream)
+
+    def close(self):
+        if getattr(self, "handle", None) and self.handle.value:
+            lib.ist_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # --- calls -----------------------------------------------------------------------------
+    def bind_weights(self, W: Sequence[torch.Tensor], b: Sequence[torch.Tensor]):
+        assert len(W) == self.t and len(b) == self.t
+        for l in range(self.t):
+            assert W[l].is_cuda and W[l].dtype == torch.float32 and W[l].is_contiguous()
+            assert tuple(W[l].shape) == (self.layer_dims[l], self.layer_dims[l + 1])
+            assert b[l].is_cuda and b[l].dtype == torch.float32 and tuple(b[l].shape) == (self.layer_dims[l + 1],)
+        self.W, self.b = list(W), list(b)
+        Wp = (ctypes.c_void_p * self.t)(*[w.data_ptr() for w in W])
+        bp = (ctypes.c_void_p * self.t)(*[v.data_ptr() for v in b])
+        _check(self.handle, lib.ist_bind_weights(self.handle, Wp, bp))
+
+    def partition(self, seed: int):
+        _check(self.handle, lib.ist_partition(self.handle, ctypes.c_uint64(seed & (2 ** 64 - 1))))
+
+    def get_partition(self, hidden_layer: int):
+        idx = torch.empty(self.layer_dims[hidden_layer], dtype=torch.int32, device=self.device)
+        off = torch.empty(self.S + 1, dtype=torch.int32, device=self.device)
+        _check(self.handle, lib.ist_get_partition(self.handle, hidden_layer, idx.data_ptr(), off.data_ptr()))
+        return idx, off
+
+    def _count(self, l: int, s: int) -> int:
+        if l == 0 or l == self.t:
+            return self.layer_dims[l]
+        N = self.layer_dims[l]
+        return N // self.S + (1 if s < N % self.S else 0)
+
+    def get_subnet_params(self, layer: int, s: int):
+        Wt = torch.empty((self._count(layer - 1, s), self._count(layer, s)), dtype=torch.float32, device=self.device)
+        bt = torch.empty(self._count(layer, s), dtype=torch.float32, device=self.device)
+        _check(self.handle, lib.ist_get_subnet_params(self.handle, layer, s, Wt.data_ptr(), bt.data_ptr()))
+        return Wt, bt
+
+    def local_steps(self, X, y: torch.Tensor, lr: float, K: int, batch: int,
+                    stride_subnet: Optional[int] = None, stride_step: Optional[int] = None,
+                    loss_out: Optional[torch.Tensor] = None, want_loss: bool = True):
+        """X rows ordered [S][K][batch] by default (stride_subnet = K*batch, stride_step = batch)."""
+        if stride_subnet is None:
+            stride_subnet = K * batch
+        if stride_step is None:
+            stride_step = batch
+        inp, keep = make_input(X, batch, stride_subnet, stride_step)
+        assert y.is_cuda and y.dtype == torch.int32 and y.is_contiguous()
+        if loss_out is None and want_loss:
+            loss_out = torch.empty(self.S * K, dtype=torch.float32, device=self.device)
+        _check(self.handle, lib.ist_local_steps(self.handle, ctypes.byref(inp), y.data_ptr(),
+                                                ctypes.c_float(lr), K, _ptr(loss_out)))
+        return loss_out.view(self.S, K) if loss_out is not None else None
+
+    def reassemble(self):
+        _check(self.handle, lib.ist_reassemble(self.handle))
+
+    def eval(self, X, y: torch.Tensor, n: int):
+        inp, keep = make_input(X, 0, 0, 0)
+        loss = torch.empty(1, dtype=torch.float32, device=self.device)
+        correct = torch.empty(1, dtype=torch.int64, device=self.device)
+        _check(self.handle, lib.ist_eval(self.handle, ctypes.byref(inp), y.data_ptr(), n,
+                                         loss.data_ptr(), correct.data_ptr()))
+        return loss, correct
+
+    def sync_status(self):
+        _check(self.handle, lib.ist_sync_status(self.handle))
+
+    def profile(self, enable: bool):
+        _check(self.handle, lib.ist_profile(self.handle, int(bool(enable))))
+
+    def profile_read(self):
+        """{class name: (kernels launched, device milliseconds)} since profiling was enabled."""
+        out = {}
+        for k, name in enumerate(KERNEL_CLASSES):
+            n, ms = ctypes.c_int64(), ctypes.c_double()
+            _check(self.handle, lib.ist_profile_read(self.handle, k, ctypes.byref(n), ctypes.byref(ms)))
+            out[name] = (int(n.value), float(ms.value))
+        return out
+
+    def kernel_launches(self) -> int:
+        return int(lib.ist_kernel_launches(self.handle))
+
+    # --- one whole round ---------------------------------------------------------------------
+    def round(self, seed: int, X, y, lr: float, K: int, batch: int, loss_out=None, want_loss=True):
+        self.partition(seed)
+        loss = self.local_steps(X, y, lr, K, batch, loss_out=loss_out, want_loss=want_loss)
+        self.reassemble()
+        return loss

@@ -1,0 +1,621 @@
+// C-ABI boundary of the IST library (see include/ist.h): argument checks, workspace carving,
+// the call-order state machine, and the sequence of kernels each call enqueues.  Every step
+// of a round runs in this library's kernels; the host only validates and enqueues.
+#include "../../include/ist.h"
+
+#include <cstdarg>
+#include <cstdio>
+#include <string>
+#include <vector>
+
+#include "kernels.h"
+
+using namespace ist;
+
+namespace {
+
+enum State { ST_CREATED = 0, ST_BOUND = 1, ST_PARTITIONED = 2 };
+
+thread_local std::string g_create_error;
+
+struct Region {
+  size_t offset = 0;
+  template <typename T> T* at(void* base) const { return reinterpret_cast<T*>((char*)base + offset); }
+};
+
+// Placement of everything that lives in the caller's workspace blob.
+struct Plan {
+  size_t total = 0;
+  Region status, keys, rank, grp, pos, row_loss, logits, ev_a, ev_b, ev_acc;
+  std::vector<Region> idx, off;             // hidden layer l at [l]  (1..t-1)
+  std::vector<Region> master, bias, opw;    // layer l at [l]         (1..t)
+  std::vector<Region> act, delta;           // act [0..t-1], delta [1..t]
+  Region take(size_t bytes) {
+    Region r;
+    r.offset = total;
+    total += (size_t)round_up((int64_t)bytes, 256);
+    return r;
+  }
+};
+
+}  // namespace
+
+struct ist_ctx {
+  int t = 0, S = 1, precision = IST_FP32, max_batch = 0, csr = 0;
+  std::vector<int64_t> N;    // layer widths N_0..N_t
+  std::vector<int64_t> np;   // per-subnet width: N_0, ceil(N_l/S) for hidden l, N_t
+  std::vector<int64_t> ld;   // np rounded up to 8 elements (16-byte rows for bf16)
+  cudaStream_t stream = nullptr;
+  void* ws = nullptr;
+  Plan plan;
+  int state = ST_CREATED;
+  std::vector<float*> W, b;  // bound full network, index l-1
+  int64_t launches = 0;
+  uint64_t seed = 0;
+  std::string err;
+
+  // profiling: event pairs around groups of launches of one kernel class
+  struct Span { int cls; int64_t kernels; cudaEvent_t a, b; };
+  bool profiling = false;
+  std::vector<Span> spans;
+  std::vector<cudaEvent_t> event_pool;
+  cudaEvent_t new_event() {
+    cudaEvent_t e = nullptr;
+    if (!event_pool.empty()) { e = event_pool.back(); event_pool.pop_back(); }
+    else cudaEventCreate(&e);
+    return e;
+  }
+  void clear_spans() {
+    for (auto& s : spans) { event_pool.push_back(s.a); event_pool.push_back(s.b); }
+    spans.clear();
+  }
+  ~ist_ctx() {
+    clear_spans();
+    for (auto e : event_pool) cudaEventDestroy(e);
+  }
+
+  size_t esize() const { return precision == IST_BF16 ? 2 : 4; }
+  Launch launch() { return Launch{stream, &launches}; }
+  DeviceStatus* status() const { return plan.status.at<DeviceStatus>(ws); }
+  int32_t* idx(int l) const { return plan.idx[l].at<int32_t>(ws); }
+  int32_t* off(int l) const { return plan.off[l].at<int32_t>(ws); }
+  float* master(int l) const { return plan.master[l].at<float>(ws); }
+  float* bias(int l) const { return plan.bias[l].at<float>(ws); }
+  bf16* opw(int l) const { return precision == IST_BF16 ? plan.opw[l].at<bf16>(ws) : nullptr; }
+  int64_t rows_pad(int l) const { return np[l - 1]; }              // packed rows of layer l
+  int64_t slice_elems(int l) const { return np[l - 1] * ld[l]; }   // per subnet
+};
+
+namespace {
+
+// Brackets the launches made during its lifetime when profiling is on.
+struct Scope {
+  ist_ctx* c;
+  int cls;
+  int64_t before;
+  cudaEvent_t a = nullptr;
+  Scope(ist_ctx* ctx, int k) : c(ctx), cls(k), before(ctx->launches) {
+    if (c->profiling) {
+      a = c->new_event();
+      cudaEventRecord(a, c->stream);
+    }
+  }
+  ~Scope() {
+    if (a) {
+      cudaEvent_t b = c->new_event();
+      cudaEventRecord(b, c->stream);
+      c->spans.push_back({cls, c->launches - before, a, b});
+    }
+  }
+};
+
+ist_status fail(ist_ctx* c, ist_status code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (c) c->err = buf; else g_create_error = buf;
+  return code;
+}
+
+bool valid_shape(const int64_t* dims, int n_dims, int S, int precision, int max_batch, std::string* why) {
+  if (!dims || n_dims < 2 || n_dims > 64) { *why = "layer_dims must hold 2..64 entries"; return false; }
+  if (precision != IST_FP32 && precision != IST_BF16) { *why = "precision must be IST_FP32 or IST_BF16"; return false; }
+  if (max_batch < 1 || max_batch > (1 << 20)) { *why = "max_batch must be in 1..2^20"; return false; }
+  if (S < 1) { *why = "S must be >= 1"; return false; }
+  for (int i = 0; i < n_dims; ++i)
+    if (dims[i] < 1 || dims[i] > (int64_t)1 << 30) { *why = "every layer width must be in 1..2^30"; return false; }
+  if (n_dims == 2 && S != 1) { *why = "a network without hidden layers cannot be partitioned: S must be 1"; return false; }
+  for (int i = 1; i + 1 < n_dims; ++i)
+    if (S > dims[i]) { *why = "S exceeds a hidden layer's width"; return false; }
+  return true;
+}
+
+void make_plan(ist_ctx* c) {
+  Plan& p = c->plan;
+  const int t = c->t, S = c->S;
+  const int64_t Bm = c->max_batch;
+  p = Plan();
+  p.idx.resize(t + 1); p.off.resize(t + 1);
+  p.master.resize(t + 1); p.bias.resize(t + 1); p.opw.resize(t + 1);
+  p.act.resize(t + 1); p.delta.resize(t + 1);
+  p.status = p.take(sizeof(DeviceStatus));
+  int64_t maxH = 1, maxN = 0;
+  for (int l = 1; l < t; ++l) maxH = std::max(maxH, c->N[l]);
+  for (int l = 0; l <= t; ++l) maxN = std::max(maxN, c->N[l]);
+  p.keys = p.take(maxH * 8);
+  p.rank = p.take(maxH * 4);
+  p.grp = p.take(maxH * 4);
+  p.pos = p.take(maxH * 4);
+  for (int l = 1; l < t; ++l) {
+    p.idx[l] = p.take(c->N[l] * 4);
+    p.off[l] = p.take((S + 1) * 4);
+  }
+  for (int l = 1; l <= t; ++l) {
+    p.master[l] = p.take((size_t)S * c->slice_elems(l) * 4);
+    p.bias[l] = p.take((size_t)S * c->ld[l] * 4);
+    if (c->precision == IST_BF16) p.opw[l] = p.take((size_t)S * c->slice_elems(l) * 2);
+  }
+  const size_t es = c->esize();
+  if (!c->csr) p.act[0] = p.take((size_t)S * Bm * c->ld[0] * es);   // staging of fp32 inputs
+  for (int l = 1; l < t; ++l) p.act[l] = p.take((size_t)S * Bm * c->ld[l] * es);
+  for (int l = 1; l <= t; ++l) p.delta[l] = p.take((size_t)S * Bm * c->ld[l] * es);
+  p.logits = p.take((size_t)S * Bm * c->ld[t] * 4);
+  p.row_loss = p.take((size_t)S * Bm * 4);
+  p.ev_a = p.take((size_t)Bm * maxN * 4);
+  p.ev_b = p.take((size_t)Bm * maxN * 4);
+  p.ev_acc = p.take(64);
+}
+
+void fill_shape(ist_ctx* c, const int64_t* dims, int n_dims, int S, int precision, int max_batch, int csr) {
+  c->t = n_dims - 1;
+  c->S = S;
+  c->precision = precision;
+  c->max_batch = max_batch;
+  c->csr = csr ? 1 : 0;
+  c->N.assign(dims, dims + n_dims);
+  c->np.resize(n_dims);
+  c->ld.resize(n_dims);
+  for (int l = 0; l <= c->t; ++l) {
+    c->np[l] = (l == 0 || l == c->t) ? dims[l] : ceil_div(dims[l], S);
+    c->ld[l] = round_up(c->np[l], 8);
+  }
+  make_plan(c);
+}
+
+ist_status cuda_fail(ist_ctx* c, cudaError_t e, const char* what) {
+  return fail(c, IST_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define IST_CUDA(c, call)                                   \
+  do {                                                      \
+    cudaError_t e_ = (call);                                \
+    if (e_ != cudaSuccess) return cuda_fail(c, e_, #call);  \
+  } while (0)
+
+uint64_t splitmix64_next(uint64_t* state) {
+  uint64_t z = (*state += 0x9E3779B97F4A7C15ull);
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+// Slice map of layer l (1..t): rows follow hidden layer l-1's partition, columns layer l's.
+SliceMap slice_map(const ist_ctx* c, int l) {
+  SliceMap m{};
+  const bool rows_indexed = l > 1, cols_indexed = l < c->t;
+  m.row_idx = rows_indexed ? c->idx(l - 1) : nullptr;
+  m.row_off = rows_indexed ? c->off(l - 1) : nullptr;
+  m.col_idx = cols_indexed ? c->idx(l) : nullptr;
+  m.col_off = cols_indexed ? c->off(l) : nullptr;
+  m.full_rows = c->N[l - 1];
+  m.full_cols = c->N[l];
+  m.rows_pad = c->np[l - 1];
+  m.ld = c->ld[l];
+  return m;
+}
+
+SliceMap bias_map(const ist_ctx* c, int l) {
+  SliceMap m{};
+  const bool cols_indexed = l < c->t;
+  m.col_idx = cols_indexed ? c->idx(l) : nullptr;
+  m.col_off = cols_indexed ? c->off(l) : nullptr;
+  m.full_rows = 1;
+  m.full_cols = c->N[l];
+  m.rows_pad = 1;
+  m.ld = c->ld[l];
+  return m;
+}
+
+ist_status check_input(ist_ctx* c, const ist_input* X, const int32_t* y, bool training) {
+  if (!X || !y) return fail(c, IST_ERR_ARG, "X and y_dev must not be null");
+  if (X->kind != IST_X_DENSE_F32 && X->kind != IST_X_DENSE_BF16 && X->kind != IST_X_CSR)
+    return fail(c, IST_ERR_ARG, "unknown input kind %d", X->kind);
+  if ((X->kind == IST_X_CSR) != (c->csr != 0))
+    return fail(c, IST_ERR_ARG, "input kind does not match input_is_csr given to ist_create");
+  if (X->kind == IST_X_CSR) {
+    if (!X->row_ptr || !X->col || !X->val) return fail(c, IST_ERR_ARG, "CSR input needs row_ptr, col and val");
+  } else {
+    if (!X->dense) return fail(c, IST_ERR_ARG, "dense input pointer is null");
+    if (X->kind == IST_X_DENSE_BF16) {
+      if (c->precision != IST_BF16 && training)
+        return fail(c, IST_ERR_UNSUPPORTED, "bf16 inputs need a bf16-precision context");
+      if (c->N[0] % 8 != 0 || ((uintptr_t)X->dense & 15))
+        return fail(c, IST_ERR_ARG, "bf16 rows need N_0 %% 8 == 0 and a 16-byte aligned base");
+    }
+  }
+  if (training) {
+    if (X->batch < 1 || X->batch > c->max_batch)
+      return fail(c, IST_ERR_ARG, "batch %d outside 1..max_batch (%d)", X->batch, c->max_batch);
+    if (X->stride_subnet < 0 || X->stride_step < 0) return fail(c, IST_ERR_ARG, "negative row stride");
+  }
+  return IST_OK;
+}
+
+// ---- grouped GEMM dispatch ------------------------------------------------------------------
+template <typename T>
+void gemm(ist_ctx* c, const GemmArgs<T>& a) {
+  gemm_simt<T>(c->launch(), a);
+}
+
+// One call of ist_local_steps in operand type T.
+template <typename T>
+ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, float lr, int K,
+                           float* loss_out) {
+  const int t = c->t, S = c->S, B = X->batch;
+  const int64_t Bm = c->max_batch;
+  const bool bf = c->precision == IST_BF16;
+  auto act = [&](int l) { return c->plan.act[l].at<T>(c->ws); };
+  auto delta = [&](int l) { return c->plan.delta[l].at<T>(c->ws); };
+  auto weights = [&](int l) -> const T* {       // operand copy of layer l's slices
+    return bf ? reinterpret_cast<const T*>(c->opw(l)) : reinterpret_cast<const T*>(c->master(l));
+  };
+  float* logits = c->plan.logits.at<float>(c->ws);
+  float* row_loss = c->plan.row_loss.at<float>(c->ws);
+  DeviceStatus* st = c->status();
+  Launch L = c->launch();
+
+  for (int k = 0; k < K; ++k) {
+    const int64_t row0 = (int64_t)k * X->stride_step;
+    // ---- layer-0 activations ---------------------------------------------------------------
+    const T* a0 = nullptr;
+    int64_t a0_ld = 0, a0_sg = 0;
+    if (X->kind != IST_X_CSR) {
+      const bool direct = (X->kind == IST_X_DENSE_BF16) == bf;
+      if (direct) {
+        a0 = reinterpret_cast<const T*>(X->dense) + row0 * c->N[0];
+        a0_ld = c->N[0];
+        a0_sg = X->stride_subnet * c->N[0];
+      } else {  // fp32 rows into a bf16 context: round into the staging buffer
+        Scope sc(c, IST_K_STAGE);
+        stage_rows<T>(L, reinterpret_cast<const float*>(X->dense) + row0 * c->N[0], c->N[0],
+                      X->stride_subnet, S, B, act(0), c->ld[0], Bm * c->ld[0]);
+        a0 = act(0);
+        a0_ld = c->ld[0];
+        a0_sg = Bm * c->ld[0];
+      }
+    }
+    auto in_ptr = [&](int l) { return l == 0 ? a0 : act(l); };
+    auto in_ld = [&](int l) { return l == 0 ? a0_ld : c->ld[l]; };
+    auto in_sg = [&](int l) { return l == 0 ? a0_sg : Bm * c->ld[l]; };
+
+    // ---- forward ---------------------------------------------------------------------------
+    for (int l = 1; l <= t; ++l) {
+      if (l == 1 && X->kind == IST_X_CSR && t > 1) {
+        Scope sc(c, IST_K_SPMM);
+        spmm_forward<T, T>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
+                           weights(1), c->ld[1], c->slice_elems(1), c->bias(1), c->ld[1],
+                           (int)c->np[1], act(1), c->ld[1], Bm * c->ld[1], st);
+        continue;
+      }
+      GemmArgs<T> g{};
+      g.M = B; g.N = (int)c->np[l]; g.K = (int)c->np[l - 1]; g.G = S;
+      g.A = in_ptr(l - 1); g.a_sm = in_ld(l - 1); g.a_sk = 1; g.a_sg = in_sg(l - 1);
+      g.B = weights(l); g.b_sn = 1; g.b_sk = c->ld[l]; g.b_sg = c->slice_elems(l);
+      g.bias = c->bias(l); g.bias_sg = c->ld[l];
+      if (l < t) {
+        g.epi = EPI_BIAS_RELU;
+        g.out = act(l); g.out_ld = c->ld[l]; g.out_sg = Bm * c->ld[l];
+      } else {
+        g.epi = EPI_BIAS_F32;
+        g.outf = logits; g.outf_ld = c->ld[t]; g.outf_sg = Bm * c->ld[t];
+      }
+      Scope sc(c, IST_K_FWD);
+      gemm<T>(c, g);
+    }
+    // ---- loss and its gradient -------------------------------------------------------------
+    {
+      Scope sc(c, IST_K_LOSS);
+      softmax_xent<T>(L, logits, c->ld[t], Bm * c->ld[t], S, B, (int)c->N[t], y + row0,
+                      X->stride_subnet, delta(t), c->ld[t], Bm * c->ld[t], row_loss, st);
+      if (loss_out) loss_reduce(L, row_loss, S, B, loss_out, K, k);
+    }
+    // ---- backward + SGD, last layer first.  delta_{l-1} is taken before W_l is updated. -----
+    for (int l = t; l >= 1; --l) {
+      if (l > 1) {
+        GemmArgs<T> g{};
+        g.M = B; g.N = (int)c->np[l - 1]; g.K = (int)c->np[l]; g.G = S;
+        g.A = delta(l); g.a_sm = c->ld[l]; g.a_sk = 1; g.a_sg = Bm * c->ld[l];
+        g.B = weights(l); g.b_sn = c->ld[l]; g.b_sk = 1; g.b_sg = c->slice_elems(l);
+        g.epi = EPI_RELU_MASK;
+        g.mask = act(l - 1); g.mask_ld = c->ld[l - 1]; g.mask_sg = Bm * c->ld[l - 1];
+        g.out = delta(l - 1); g.out_ld = c->ld[l - 1]; g.out_sg = Bm * c->ld[l - 1];
+        Scope sc(c, IST_K_DX);
+        gemm<T>(c, g);
+      }
+      {
+        Scope sc(c, IST_K_BIAS_SGD);
+        bias_sgd<T>(L, delta(l), c->ld[l], Bm * c->ld[l], S, B, (int)c->np[l], c->bias(l), c->ld[l], lr);
+      }
+      if (l == 1 && X->kind == IST_X_CSR && t > 1) {
+        Scope sc(c, IST_K_SPMM);
+        spmm_backward_sgd<T>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
+                             delta(1), c->ld[1], Bm * c->ld[1], (int)c->np[1], c->master(1), c->opw(1),
+                             c->ld[1], c->slice_elems(1), lr);
+        continue;
+      }
+      GemmArgs<T> g{};
+      g.M = (int)c->np[l - 1]; g.N = (int)c->np[l]; g.K = B; g.G = S;
+      g.A = in_ptr(l - 1); g.a_sm = 1; g.a_sk = in_ld(l - 1); g.a_sg = in_sg(l - 1);
+      g.B = delta(l); g.b_sn = 1; g.b_sk = c->ld[l]; g.b_sg = Bm * c->ld[l];
+      g.epi = EPI_SGD;
+      g.outf = c->master(l); g.outf_ld = c->ld[l]; g.outf_sg = c->slice_elems(l);
+      g.opw = c->opw(l);
+      g.lr = lr;
+      Scope sc(c, IST_K_DW_SGD);
+      gemm<T>(c, g);
+    }
+  }
+  IST_CUDA(c, cudaGetLastError());
+  return IST_OK;
+}
+
+}  // namespace
+
+// ================================= public entry points =======================================
+
+extern "C" size_t ist_workspace_bytes(const int64_t* layer_dims, int n_dims, int S, int precision,
+                                      int max_batch, int input_is_csr) {
+  std::string why;
+  if (!valid_shape(layer_dims, n_dims, S, precision, max_batch, &why)) {
+    g_create_error = why;
+    return 0;
+  }
+  ist_ctx tmp;
+  fill_shape(&tmp, layer_dims, n_dims, S, precision, max_batch, input_is_csr);
+  return tmp.plan.total;
+}
+
+extern "C" ist_status ist_create(ist_ctx** out, const int64_t* layer_dims, int n_dims, int S,
+                                 int precision, int max_batch, int input_is_csr, void* workspace_dev,
+                                 size_t workspace_bytes, void* cuda_stream) {
+  if (!out) return fail(nullptr, IST_ERR_ARG, "out must not be null");
+  std::string why;
+  if (!valid_shape(layer_dims, n_dims, S, precision, max_batch, &why))
+    return fail(nullptr, IST_ERR_ARG, "%s", why.c_str());
+  if (input_is_csr && n_dims < 3)
+    return fail(nullptr, IST_ERR_UNSUPPORTED, "CSR inputs need at least one hidden layer");
+  ist_ctx* c = new ist_ctx();
+  fill_shape(c, layer_dims, n_dims, S, precision, max_batch, input_is_csr);
+  if (!workspace_dev || ((uintptr_t)workspace_dev & 255)) {
+    delete c;
+    return fail(nullptr, IST_ERR_WORKSPACE, "workspace must be a 256-byte aligned device pointer");
+  }
+  if (workspace_bytes < c->plan.total) {
+    size_t need = c->plan.total;
+    delete c;
+    return fail(nullptr, IST_ERR_WORKSPACE, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
+  }
+  c->ws = workspace_dev;
+  c->stream = (cudaStream_t)cuda_stream;
+  cudaError_t e = cudaMemsetAsync(workspace_dev, 0, c->plan.total, c->stream);
+  if (e != cudaSuccess) {
+    delete c;
+    return fail(nullptr, IST_ERR_CUDA, "clearing the workspace: %s", cudaGetErrorString(e));
+  }
+  *out = c;
+  return IST_OK;
+}
+
+extern "C" ist_status ist_bind_weights(ist_ctx* c, float* const* W_dev, float* const* b_dev) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state == ST_PARTITIONED) return fail(c, IST_ERR_STATE, "cannot rebind between ist_partition and ist_reassemble");
+  if (!W_dev || !b_dev) return fail(c, IST_ERR_ARG, "W_dev and b_dev must not be null");
+  for (int l = 0; l < c->t; ++l) {
+    if (!W_dev[l] || !b_dev[l]) return fail(c, IST_ERR_ARG, "layer %d: null weight or bias pointer", l + 1);
+    if (((uintptr_t)W_dev[l] & 15) || ((uintptr_t)b_dev[l] & 3))
+      return fail(c, IST_ERR_ARG, "layer %d: weights must be 16-byte aligned", l + 1);
+  }
+  c->W.assign(W_dev, W_dev + c->t);
+  c->b.assign(b_dev, b_dev + c->t);
+  c->state = ST_BOUND;
+  return IST_OK;
+}
+
+extern "C" ist_status ist_partition(ist_ctx* c, uint64_t seed) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state != ST_BOUND) return fail(c, IST_ERR_STATE, "ist_partition needs bound weights and no partition in place");
+  Launch L = c->launch();
+  const int t = c->t, S = c->S;
+  c->seed = seed;
+  uint64_t round_state = seed;
+  for (int l = 1; l < t; ++l) {
+    Scope sc(c, IST_K_PARTITION);
+    uint64_t layer_seed = splitmix64_next(&round_state);
+    partition_layer(L, layer_seed, (int)c->N[l], S, c->plan.keys.at<uint64_t>(c->ws),
+                    c->plan.rank.at<int32_t>(c->ws), c->plan.grp.at<int32_t>(c->ws),
+                    c->plan.pos.at<int32_t>(c->ws), c->idx(l), c->off(l), c->status());
+  }
+  for (int l = 1; l <= t; ++l) {
+    Scope sc(c, IST_K_GATHER);
+    gather_slices(L, c->W[l - 1], slice_map(c, l), S, c->master(l), c->opw(l));
+    gather_slices(L, c->b[l - 1], bias_map(c, l), S, c->bias(l), nullptr);
+  }
+  IST_CUDA(c, cudaGetLastError());
+  c->state = ST_PARTITIONED;
+  return IST_OK;
+}
+
+extern "C" ist_status ist_get_partition(ist_ctx* c, int hidden_layer, int32_t* idx_out_dev,
+                                        int32_t* off_out_dev) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state != ST_PARTITIONED) return fail(c, IST_ERR_STATE, "no partition in place");
+  if (hidden_layer < 1 || hidden_layer >= c->t) return fail(c, IST_ERR_ARG, "hidden_layer outside 1..t-1");
+  if (idx_out_dev)
+    IST_CUDA(c, cudaMemcpyAsync(idx_out_dev, c->idx(hidden_layer), c->N[hidden_layer] * 4,
+                                cudaMemcpyDeviceToDevice, c->stream));
+  if (off_out_dev)
+    IST_CUDA(c, cudaMemcpyAsync(off_out_dev, c->off(hidden_layer), (c->S + 1) * 4,
+                                cudaMemcpyDeviceToDevice, c->stream));
+  return IST_OK;
+}
+
+extern "C" ist_status ist_get_subnet_params(ist_ctx* c, int layer, int s, float* W_out_dev,
+                                            float* b_out_dev) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state != ST_PARTITIONED) return fail(c, IST_ERR_STATE, "no partition in place");
+  if (layer < 1 || layer > c->t || s < 0 || s >= c->S) return fail(c, IST_ERR_ARG, "layer or subnet out of range");
+  auto count = [&](int l) -> int64_t {   // |G_l^s| (balanced split), full width at the ends
+    if (l == 0 || l == c->t) return c->N[l];
+    return c->N[l] / c->S + (s < c->N[l] % c->S ? 1 : 0);
+  };
+  Launch L = c->launch();
+  if (W_out_dev)
+    copy_out_slice(L, c->master(layer) + (int64_t)s * c->slice_elems(layer), c->ld[layer],
+                   count(layer - 1), count(layer), W_out_dev);
+  if (b_out_dev)
+    copy_out_slice(L, c->bias(layer) + (int64_t)s * c->ld[layer], c->ld[layer], 1, count(layer), b_out_dev);
+  IST_CUDA(c, cudaGetLastError());
+  return IST_OK;
+}
+
+extern "C" ist_status ist_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y_dev, float lr,
+                                      int K, float* loss_out_dev) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state != ST_PARTITIONED) return fail(c, IST_ERR_STATE, "ist_local_steps needs a partition in place");
+  if (K < 1) return fail(c, IST_ERR_ARG, "K must be >= 1");
+  if (!(lr == lr)) return fail(c, IST_ERR_ARG, "lr is NaN");
+  ist_status s = check_input(c, X, y_dev, true);
+  if (s != IST_OK) return s;
+  if (c->precision == IST_BF16) return run_local_steps<bf16>(c, X, y_dev, lr, K, loss_out_dev);
+  return run_local_steps<float>(c, X, y_dev, lr, K, loss_out_dev);
+}
+
+extern "C" ist_status ist_reassemble(ist_ctx* c) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state != ST_PARTITIONED) return fail(c, IST_ERR_STATE, "ist_reassemble needs a partition in place");
+  Launch L = c->launch();
+  const int t = c->t, S = c->S;
+  for (int l = 1; l <= t; ++l) {
+    Scope sc(c, IST_K_SCATTER);
+    scatter_slices(L, c->W[l - 1], slice_map(c, l), S, c->master(l));
+    if (l < t) scatter_slices(L, c->b[l - 1], bias_map(c, l), S, c->bias(l));
+  }
+  {
+    Scope sc(c, IST_K_SCATTER);
+    scatter_mean_bias(L, c->b[t - 1], c->N[t], S, c->bias(t), c->ld[t]);
+  }
+  IST_CUDA(c, cudaGetLastError());
+  c->state = ST_BOUND;
+  return IST_OK;
+}
+
+extern "C" ist_status ist_eval(ist_ctx* c, const ist_input* X, const int32_t* y_dev, int64_t n,
+                               float* mean_loss_out_dev, int64_t* n_correct_out_dev) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state != ST_BOUND) return fail(c, IST_ERR_STATE, "ist_eval needs bound weights and no partition in place");
+  if (n < 1) return fail(c, IST_ERR_ARG, "n must be >= 1");
+  if (!mean_loss_out_dev || !n_correct_out_dev) return fail(c, IST_ERR_ARG, "output pointers must not be null");
+  ist_status s = check_input(c, X, y_dev, false);
+  if (s != IST_OK) return s;
+  if (X->kind == IST_X_DENSE_BF16) return fail(c, IST_ERR_UNSUPPORTED, "ist_eval takes fp32 or CSR rows");
+  Launch L = c->launch();
+  const int t = c->t;
+  float* buf[2] = {c->plan.ev_a.at<float>(c->ws), c->plan.ev_b.at<float>(c->ws)};
+  double* loss_sum = c->plan.ev_acc.at<double>(c->ws);
+  long long* correct = reinterpret_cast<long long*>(loss_sum + 1);
+  IST_CUDA(c, cudaMemsetAsync(loss_sum, 0, 16, c->stream));
+  Scope sc(c, IST_K_EVAL);
+  for (int64_t r0 = 0; r0 < n; r0 += c->max_batch) {
+    const int rows = (int)std::min<int64_t>(c->max_batch, n - r0);
+    const float* in = nullptr;
+    int64_t in_ld = 0;
+    int cur = 0;
+    for (int l = 1; l <= t; ++l) {
+      float* o = buf[cur];
+      if (l == 1 && X->kind == IST_X_CSR) {
+        spmm_forward<float, float>(L, X->row_ptr, X->col, X->val, r0, 0, 1, rows, c->N[0], c->W[0], c->N[1],
+                                   0, c->b[0], 0, (int)c->N[1], o, c->N[1], 0, c->status());
+      } else {
+        GemmArgs<float> g{};
+        g.M = rows; g.N = (int)c->N[l]; g.K = (int)c->N[l - 1]; g.G = 1;
+        if (l == 1) { g.A = reinterpret_cast<const float*>(X->dense) + r0 * c->N[0]; g.a_sm = c->N[0]; }
+        else { g.A = in; g.a_sm = in_ld; }
+        g.a_sk = 1;
+        g.B = c->W[l - 1]; g.b_sn = 1; g.b_sk = c->N[l];
+        g.bias = c->b[l - 1];
+        if (l < t) { g.epi = EPI_BIAS_RELU; g.out = o; g.out_ld = c->N[l]; }
+        else { g.epi = EPI_BIAS_F32; g.outf = o; g.outf_ld = c->N[l]; }
+        gemm_simt<float>(L, g);
+      }
+      in = o;
+      in_ld = c->N[l];
+      cur ^= 1;
+    }
+    eval_rows(L, in, in_ld, rows, (int)c->N[t], y_dev + r0, loss_sum, correct, c->status());
+  }
+  eval_finalize(L, loss_sum, correct, n, mean_loss_out_dev, n_correct_out_dev);
+  IST_CUDA(c, cudaGetLastError());
+  return IST_OK;
+}
+
+extern "C" ist_status ist_sync_status(ist_ctx* c) {
+  if (!c) return IST_ERR_ARG;
+  DeviceStatus h{};
+  IST_CUDA(c, cudaMemcpyAsync(&h, c->status(), sizeof h, cudaMemcpyDeviceToHost, c->stream));
+  IST_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (h.code != 0) {
+    static const char* sites[] = {"", "label out of range", "CSR column out of range",
+                                  "partition index out of range", "tensor-core pipeline wait expired",
+                                  "CSR row_ptr not monotone"};
+    const char* w = (h.site >= 0 && h.site <= 5) ? sites[h.site] : "?";
+    return fail(c, (ist_status)h.code, "device status %d: %s (detail %lld)", h.code, w, h.detail);
+  }
+  return IST_OK;
+}
+
+extern "C" ist_status ist_profile(ist_ctx* c, int enable) {
+  if (!c) return IST_ERR_ARG;
+  IST_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (enable) c->clear_spans();
+  c->profiling = enable != 0;
+  return IST_OK;
+}
+
+extern "C" ist_status ist_profile_read(ist_ctx* c, int kernel_class, int64_t* launches_out_host,
+                                       double* ms_out_host) {
+  if (!c) return IST_ERR_ARG;
+  if (kernel_class < 0 || kernel_class >= IST_K_COUNT) return fail(c, IST_ERR_ARG, "unknown kernel class");
+  IST_CUDA(c, cudaStreamSynchronize(c->stream));
+  int64_t n = 0;
+  double ms = 0.0;
+  for (auto& s : c->spans) {
+    if (s.cls != kernel_class) continue;
+    float t = 0.f;
+    IST_CUDA(c, cudaEventElapsedTime(&t, s.a, s.b));
+    ms += t;
+    n += s.kernels;
+  }
+  if (launches_out_host) *launches_out_host = n;
+  if (ms_out_host) *ms_out_host = ms;
+  return IST_OK;
+}
+
+extern "C" int64_t ist_kernel_launches(const ist_ctx* c) { return c ? c->launches : 0; }
+
+extern "C" const char* ist_last_error(const ist_ctx* c) {
+  return c ? c->err.c_str() : g_create_error.c_str();
+}
+
+extern "C" void ist_destroy(ist_ctx* c) { delete c; }

@@ -1,0 +1,106 @@
+// Host-side launchers of the IST library's kernels (internal; the public boundary is ist.h).
+#pragma once
+
+#include "common.cuh"
+
+namespace ist {
+
+struct Launch {
+  cudaStream_t stream;
+  int64_t* counter;  // host counter of kernels launched
+  void count(int n = 1) const { if (counter) *counter += n; }
+};
+
+// ---- partition.cu -----------------------------------------------------------------------
+// Balanced random partition of {0..N-1} into S groups from SplitMix64 keys (see ist.h).
+// Scratch: keys [N] u64, rank [N] i32, grp [N] i32, pos [N] i32.  Outputs: idx [N], off [S+1].
+void partition_layer(const Launch& L, uint64_t layer_seed, int N, int S, uint64_t* keys,
+                     int32_t* rank, int32_t* grp, int32_t* pos, int32_t* idx, int32_t* off,
+                     DeviceStatus* st);
+
+// ---- gather_scatter.cu ------------------------------------------------------------------
+// A slice map describes how packed element (s, i, j) of a layer relates to the full matrix:
+// full row = row_idx ? row_idx[row_off[s] + i] : i, full col likewise.
+struct SliceMap {
+  const int32_t* row_idx;
+  const int32_t* row_off;
+  const int32_t* col_idx;
+  const int32_t* col_off;
+  int64_t full_rows, full_cols;  // N_{l-1}, N_l (row stride of the full matrix = full_cols)
+  int64_t rows_pad, ld;          // packed slice: [S][rows_pad][ld]
+};
+void gather_slices(const Launch& L, const float* W, const SliceMap& m, int S, float* master,
+                   bf16* opw);
+void scatter_slices(const Launch& L, float* W, const SliceMap& m, int S, const float* master);
+// b[j] += (sum_s (packed[s][j] - b[j])) / S for the output bias.
+void scatter_mean_bias(const Launch& L, float* b, int64_t n, int S, const float* packed,
+                       int64_t ld);
+// Dense copy-out of a packed slice (ist_get_subnet_params).
+void copy_out_slice(const Launch& L, const float* packed, int64_t ld, int64_t rows, int64_t cols,
+                    float* out);
+
+// ---- grouped GEMM -----------------------------------------------------------------------
+// C[g](m, n) = sum_k A[g](m, k) * B[g](n, k), fp32 accumulation, followed by an epilogue.
+enum Epilogue : int {
+  EPI_BIAS_RELU = 0,  // out = T(max(C + bias[n], 0))
+  EPI_BIAS_F32 = 1,   // outf = C + bias[n]                     (logits)
+  EPI_RELU_MASK = 2,  // out = T(mask > 0 ? C : 0)              (delta through ReLU)
+  EPI_SGD = 3,        // outf -= lr * C; opw = bf16(outf) if opw (fused weight update)
+  EPI_STORE = 4       // out = T(C)
+};
+
+template <typename T>
+struct GemmArgs {
+  int M, N, K, G;
+  const T* A; int64_t a_sm, a_sk, a_sg;
+  const T* B; int64_t b_sn, b_sk, b_sg;
+  int epi;
+  const float* bias; int64_t bias_sg;
+  T* out; int64_t out_ld, out_sg;
+  float* outf; int64_t outf_ld, outf_sg;
+  const T* mask; int64_t mask_ld, mask_sg;
+  bf16* opw;
+  float lr;
+};
+template <typename T> void gemm_simt(const Launch& L, const GemmArgs<T>& a);
+
+// ---- rowops.cu --------------------------------------------------------------------------
+// Row-wise softmax cross-entropy of logits [G][B][ld] against labels; writes
+// delta = (softmax - onehot)/B (zero in columns Nt..ld_d) and row_loss [G][B].
+template <typename T>
+void softmax_xent(const Launch& L, const float* logits, int64_t ld, int64_t sg, int G, int B, int Nt,
+                  const int32_t* y, int64_t y_sg, T* delta, int64_t ld_d, int64_t sg_d,
+                  float* row_loss, DeviceStatus* st);
+// loss_out[g * out_stride + k] = (1/B) sum_b row_loss[g][b]  (fixed summation order)
+void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
+                 int64_t out_stride, int k);
+// bias[g][n] -= lr * sum_b delta[g][b][n]
+template <typename T>
+void bias_sgd(const Launch& L, const T* delta, int64_t ld, int64_t sg, int G, int B, int n,
+              float* bias, int64_t bias_sg, float lr);
+// fp32 rows -> T rows with leading dimension ld (pad columns zero), per group row offsets.
+template <typename T>
+void stage_rows(const Launch& L, const float* X, int64_t N0, int64_t group_row_stride, int G, int B,
+                T* out, int64_t ld, int64_t sg);
+// eval accumulators: loss_sum += sum of row losses, correct += #argmax hits
+void eval_rows(const Launch& L, const float* logits, int64_t ld, int rows, int Nt, const int32_t* y,
+               double* loss_sum, long long* correct, DeviceStatus* st);
+void eval_finalize(const Launch& L, const double* loss_sum, const long long* correct, int64_t n,
+                   float* mean_loss_out, int64_t* correct_out);
+
+// ---- spmm.cu ----------------------------------------------------------------------------
+// out[g][b][:] = relu(sum_nz val * P[g][col][:] + bias[g][:]) for rows r0_g + b of a CSR matrix.
+template <typename T, typename TO>
+void spmm_forward(const Launch& L, const int32_t* row_ptr, const int32_t* col, const float* val,
+                  int64_t row0, int64_t group_row_stride, int G, int B, int64_t N0, const T* P,
+                  int64_t p_ld, int64_t p_sg, const float* bias, int64_t bias_sg, int n1, TO* out,
+                  int64_t out_ld, int64_t out_sg, DeviceStatus* st);
+// master[g][col][:] -= lr * val * delta[g][b][:] over stored nonzeros (atomic adds), then
+// refresh the bf16 copy of the touched rows (opw may be null).
+template <typename T>
+void spmm_backward_sgd(const Launch& L, const int32_t* row_ptr, const int32_t* col, const float* val,
+                       int64_t row0, int64_t group_row_stride, int G, int B, int64_t N0,
+                       const T* delta, int64_t d_ld, int64_t d_sg, int n1, float* master, bf16* opw,
+                       int64_t p_ld, int64_t p_sg, float lr);
+
+}  // namespace ist

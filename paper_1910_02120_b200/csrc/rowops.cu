@@ -1,0 +1,229 @@
+// Row-wise pieces of a local SGD step that are not contractions: softmax cross-entropy and
+// its gradient, the bias update, input staging, and the evaluation reductions.
+#include "kernels.h"
+
+namespace ist {
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ float warp_max(float v) {
+  for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Block-wide reductions with a fixed tree (deterministic for a given block size).
+__device__ float block_max(float v, float* sh) {
+  v = warp_max(v);
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) sh[w] = v;
+  __syncthreads();
+  float r = l < (blockDim.x >> 5) ? sh[l] : -INFINITY;
+  return warp_max(r);
+}
+__device__ float block_sum(float v, float* sh) {
+  v = warp_sum(v);
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) sh[w] = v;
+  __syncthreads();
+  float r = l < (blockDim.x >> 5) ? sh[l] : 0.f;
+  return warp_sum(r);
+}
+
+// One CTA per row (g, b).  loss_row = log(sum exp(z - max)) + max - z[y];
+// delta = (exp(z - max)/sum - [n == y]) / B.
+template <typename T>
+__global__ void softmax_xent_kernel(const float* __restrict__ logits, int64_t ld, int64_t sg, int B,
+                                    int Nt, const int32_t* __restrict__ y, int64_t y_sg,
+                                    T* __restrict__ delta, int64_t ld_d, int64_t sg_d,
+                                    float* __restrict__ row_loss, DeviceStatus* st) {
+  __shared__ float sh[32];
+  int g = blockIdx.y, b = blockIdx.x;
+  const float* z = logits + (int64_t)g * sg + (int64_t)b * ld;
+  T* d = delta + (int64_t)g * sg_d + (int64_t)b * ld_d;
+  int label = y[(int64_t)g * y_sg + b];
+  if (label < 0 || label >= Nt) {
+    if (threadIdx.x == 0) report(st, -5, SITE_LABEL, (long long)g * B + b);
+    label = 0;
+  }
+  float mx = -INFINITY;
+  for (int n = threadIdx.x; n < Nt; n += blockDim.x) mx = fmaxf(mx, z[n]);
+  mx = block_max(mx, sh);
+  float se = 0.f;
+  for (int n = threadIdx.x; n < Nt; n += blockDim.x) se += expf(z[n] - mx);
+  se = block_sum(se, sh);
+  float inv = 1.f / se, invB = 1.f / (float)B;
+  for (int n = threadIdx.x; n < ld_d; n += blockDim.x) {
+    float v = 0.f;
+    if (n < Nt) v = (expf(z[n] - mx) * inv - (n == label ? 1.f : 0.f)) * invB;
+    d[n] = from_float<T>(v);
+  }
+  if (threadIdx.x == 0) row_loss[(int64_t)g * B + b] = logf(se) + mx - z[label];
+}
+
+__global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int B, float* loss_out,
+                                   int64_t out_stride, int k) {
+  __shared__ float sh[32];
+  int g = blockIdx.x;
+  float acc = 0.f;
+  for (int b = threadIdx.x; b < B; b += blockDim.x) acc += row_loss[(int64_t)g * B + b];
+  acc = block_sum(acc, sh);
+  if (threadIdx.x == 0) loss_out[(int64_t)g * out_stride + k] = acc / (float)B;
+}
+
+// Thread per column; 8 row-lanes per column reduce through shared memory in fixed order.
+template <typename T>
+__global__ void bias_sgd_kernel(const T* __restrict__ delta, int64_t ld, int64_t sg, int B, int n,
+                                float* bias, int64_t bias_sg, float lr) {
+  __shared__ float part[8][33];
+  int g = blockIdx.y;
+  int col = blockIdx.x * 32 + threadIdx.x;
+  float acc = 0.f;
+  if (col < n) {
+    const T* d = delta + (int64_t)g * sg + col;
+    for (int b = threadIdx.y; b < B; b += 8) acc += to_float(d[(int64_t)b * ld]);
+  }
+  part[threadIdx.y][threadIdx.x] = acc;
+  __syncthreads();
+  if (threadIdx.y == 0 && col < n) {
+    float s = 0.f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) s += part[u][threadIdx.x];
+    bias[(int64_t)g * bias_sg + col] -= lr * s;
+  }
+}
+
+template <typename T>
+__global__ void stage_rows_kernel(const float* __restrict__ X, int64_t N0, int64_t group_row_stride,
+                                  int B, T* __restrict__ out, int64_t ld, int64_t sg) {
+  int g = blockIdx.z, b = blockIdx.y;
+  int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= ld) return;
+  float v = j < N0 ? X[((int64_t)g * group_row_stride + b) * N0 + j] : 0.f;
+  out[(int64_t)g * sg + (int64_t)b * ld + j] = from_float<T>(v);
+}
+
+__global__ void eval_rows_kernel(const float* __restrict__ logits, int64_t ld, int rows, int Nt,
+                                 const int32_t* __restrict__ y, double* loss_sum, long long* correct,
+                                 DeviceStatus* st) {
+  __shared__ float sh[32];
+  __shared__ int shi[32];
+  int r = blockIdx.x;
+  const float* z = logits + (int64_t)r * ld;
+  int label = y[r];
+  if (label < 0 || label >= Nt) {
+    if (threadIdx.x == 0) report(st, -5, SITE_LABEL, r);
+    label = 0;
+  }
+  float mx = -INFINITY;
+  int arg = 0x7fffffff;
+  for (int n = threadIdx.x; n < Nt; n += blockDim.x) {
+    float v = z[n];
+    if (v > mx) { mx = v; arg = n; }   // first maximum inside the thread's strided set
+  }
+  // arg-max with lowest index on ties
+  for (int o = 16; o; o >>= 1) {
+    float om = __shfl_xor_sync(0xffffffffu, mx, o);
+    int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+    if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+  }
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  if (l == 0) { sh[w] = mx; shi[w] = arg; }
+  __syncthreads();
+  if (w == 0) {
+    float m2 = l < (blockDim.x >> 5) ? sh[l] : -INFINITY;
+    int a2 = l < (blockDim.x >> 5) ? shi[l] : 0x7fffffff;
+    for (int o = 16; o; o >>= 1) {
+      float om = __shfl_xor_sync(0xffffffffu, m2, o);
+      int oa = __shfl_xor_sync(0xffffffffu, a2, o);
+      if (om > m2 || (om == m2 && oa < a2)) { m2 = om; a2 = oa; }
+    }
+    if (l == 0) { sh[0] = m2; shi[0] = a2; }
+  }
+  __syncthreads();
+  mx = sh[0];
+  arg = shi[0];
+  float se = 0.f;
+  for (int n = threadIdx.x; n < Nt; n += blockDim.x) se += expf(z[n] - mx);
+  se = block_sum(se, sh);
+  if (threadIdx.x == 0) {
+    atomicAdd(loss_sum, (double)(logf(se) + mx - z[label]));
+    if (arg == label) atomicAdd((unsigned long long*)correct, 1ull);
+  }
+}
+
+__global__ void eval_finalize_kernel(const double* loss_sum, const long long* correct, int64_t n,
+                                     float* mean_loss_out, int64_t* correct_out) {
+  *mean_loss_out = (float)(*loss_sum / (double)n);
+  *correct_out = (int64_t)*correct;
+}
+
+int row_threads(int Nt) { return Nt <= 64 ? 32 : (Nt <= 1024 ? 128 : kThreads); }
+
+}  // namespace
+
+template <typename T>
+void softmax_xent(const Launch& L, const float* logits, int64_t ld, int64_t sg, int G, int B, int Nt,
+                  const int32_t* y, int64_t y_sg, T* delta, int64_t ld_d, int64_t sg_d,
+                  float* row_loss, DeviceStatus* st) {
+  softmax_xent_kernel<T><<<dim3(B, G), row_threads(Nt), 0, L.stream>>>(
+      logits, ld, sg, B, Nt, y, y_sg, delta, ld_d, sg_d, row_loss, st);
+  L.count();
+}
+template void softmax_xent<float>(const Launch&, const float*, int64_t, int64_t, int, int, int,
+                                  const int32_t*, int64_t, float*, int64_t, int64_t, float*,
+                                  DeviceStatus*);
+template void softmax_xent<bf16>(const Launch&, const float*, int64_t, int64_t, int, int, int,
+                                 const int32_t*, int64_t, bf16*, int64_t, int64_t, float*,
+                                 DeviceStatus*);
+
+void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
+                 int64_t out_stride, int k) {
+  loss_reduce_kernel<<<G, 256, 0, L.stream>>>(row_loss, B, loss_out, out_stride, k);
+  L.count();
+}
+
+template <typename T>
+void bias_sgd(const Launch& L, const T* delta, int64_t ld, int64_t sg, int G, int B, int n,
+              float* bias, int64_t bias_sg, float lr) {
+  bias_sgd_kernel<T><<<dim3((unsigned)ceil_div(n, 32), G), dim3(32, 8), 0, L.stream>>>(
+      delta, ld, sg, B, n, bias, bias_sg, lr);
+  L.count();
+}
+template void bias_sgd<float>(const Launch&, const float*, int64_t, int64_t, int, int, int, float*,
+                              int64_t, float);
+template void bias_sgd<bf16>(const Launch&, const bf16*, int64_t, int64_t, int, int, int, float*,
+                             int64_t, float);
+
+template <typename T>
+void stage_rows(const Launch& L, const float* X, int64_t N0, int64_t group_row_stride, int G, int B,
+                T* out, int64_t ld, int64_t sg) {
+  stage_rows_kernel<T><<<dim3((unsigned)ceil_div(ld, 256), B, G), 256, 0, L.stream>>>(
+      X, N0, group_row_stride, B, out, ld, sg);
+  L.count();
+}
+template void stage_rows<float>(const Launch&, const float*, int64_t, int64_t, int, int, float*,
+                                int64_t, int64_t);
+template void stage_rows<bf16>(const Launch&, const float*, int64_t, int64_t, int, int, bf16*,
+                               int64_t, int64_t);
+
+void eval_rows(const Launch& L, const float* logits, int64_t ld, int rows, int Nt, const int32_t* y,
+               double* loss_sum, long long* correct, DeviceStatus* st) {
+  eval_rows_kernel<<<rows, row_threads(Nt), 0, L.stream>>>(logits, ld, rows, Nt, y, loss_sum, correct,
+                                                           st);
+  L.count();
+}
+
+void eval_finalize(const Launch& L, const double* loss_sum, const long long* correct, int64_t n,
+                   float* mean_loss_out, int64_t* correct_out) {
+  eval_finalize_kernel<<<1, 1, 0, L.stream>>>(loss_sum, correct, n, mean_loss_out, correct_out);
+  L.count();
+}
+
+}  // namespace ist

@@ -1,0 +1,61 @@
+"""Host-only checks of the C-ABI boundary: the library loads, exports every symbol the header
+declares, and rejects bad shapes before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_1910_02120_b200 import build
+    build.build()
+    from paper_1910_02120_b200 import api as a
+    return a
+
+
+def test_every_declared_symbol_is_exported(api):
+    header = open(os.path.join(ROOT, "include", "ist.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(ist_[a-z_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    assert declared == set(api.EXPORTS)
+    for name in declared:
+        assert hasattr(api.lib, name), name
+        getattr(api.lib, name)
+
+
+def test_workspace_bytes_validates_shapes(api):
+    assert api.ist_workspace_bytes([784, 1024, 10], 2, api.IST_FP32, 128) > 0
+    assert api.ist_workspace_bytes([784, 1024, 10], 0, api.IST_FP32, 128) == 0      # S < 1
+    assert api.ist_workspace_bytes([784, 10], 2, api.IST_FP32, 128) == 0            # no hidden layer, S > 1
+    assert api.ist_workspace_bytes([784, 10], 1, api.IST_FP32, 128) > 0
+    assert api.ist_workspace_bytes([8, 4, 3], 5, api.IST_FP32, 16) == 0             # S > hidden width
+    assert api.ist_workspace_bytes([8, 4, 3], 2, 7, 16) == 0                        # bad precision
+    assert api.ist_workspace_bytes([8, 4, 3], 2, api.IST_BF16, 0) == 0              # bad batch
+    assert api.ist_workspace_bytes([8, 0, 3], 1, api.IST_BF16, 4) == 0              # zero width
+
+
+def test_workspace_grows_with_shape_and_holds_the_slices(api):
+    small = api.ist_workspace_bytes([1024, 4096, 4096, 35], 4, api.IST_BF16, 256)
+    big = api.ist_workspace_bytes([3072, 16384, 16384, 10], 8, api.IST_BF16, 512)
+    assert big > small
+    # packed fp32 masters + bf16 copies of the wide config: 84.1M elements * 6 bytes at least
+    elems = 3072 * 16384 + 16384 * 16384 // 8 + 16384 * 10
+    assert big >= elems * 6
+
+
+def test_create_rejects_bad_workspace_without_a_device(api):
+    dims = (ctypes.c_int64 * 3)(8, 4, 3)
+    h = ctypes.c_void_p()
+    st = api.lib.ist_create(ctypes.byref(h), dims, 3, 2, api.IST_FP32, 4, 0, None, 0, None)
+    assert st == api.IST_ERR_WORKSPACE and not h.value
+    assert b"workspace" in api.lib.ist_last_error(None)
+    st = api.lib.ist_create(ctypes.byref(h), dims, 3, 9, api.IST_FP32, 4, 0, None, 0, None)
+    assert st == api.IST_ERR_ARG
+    st = api.lib.ist_create(ctypes.byref(h), dims, 3, 2, api.IST_FP32, 4, 0, ctypes.c_void_p(256), 16, None)
+    assert st == api.IST_ERR_WORKSPACE
+    assert api.lib.ist_partition(None, 1) == api.IST_ERR_ARG

@@ -1,0 +1,314 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, on the same seeded
+inputs: bit-exact for partitions, index maps and moved fp32 values; relative 1e-4 for one fp32
+round; 2e-2 on weights and 1e-3 absolute on mean loss for bf16.
+
+The bf16 weight *update* is also compared (a wrong gradient would pass the 2e-2 weight check
+when lr*K*|grad| << |W|).  Its tolerance is 1e-1, not the weight tolerance: bf16 rounding of
+weights and activations perturbs every hidden pre-activation by about 2^-9 of its spread, which
+flips the ReLU mask of the ~0.1-0.3 % of pre-activations that lie that close to zero; a flipped
+entry of delta is wrong by its whole magnitude, so the relative Frobenius error of delta (and
+of a^T delta) is about sqrt(flipped fraction) = 4-6 % for two hidden layers."""
+import numpy as np
+import pytest
+
+from paper_1910_02120_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+FP32_RTOL = 1e-4
+BF16_W_RTOL = 2e-2
+BF16_DW_RTOL = 1e-1
+BF16_LOSS_ATOL = 1e-3
+
+
+def _wl(name, dims, S, B, K, precision, x_dist="normal", lr=0.01, seed=77):
+    return synth.Workload(name, tuple(dims), S=S, B=B, K=K, rounds=1, precision=precision,
+                          x_dist=x_dist, lr=lr, seed=seed)
+
+
+def _parts_equal(gp, op):
+    assert len(gp) == len(op)
+    for (gi, go), (oi, oo) in zip(gp, op):
+        assert gi.dtype == np.int32 and go.dtype == np.int32
+        assert np.array_equal(gi, oi) and np.array_equal(go, oo)
+
+
+# ---------------------------------------------------------------------------------------------
+# partition: bit-exact index maps
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dims,S", [
+    ([16, 1024, 10], 2), ([8, 1000, 777, 5], 7), ([8, 4096, 4096, 35], 4), ([4, 33, 3], 1),
+    ([4, 16, 16, 3], 16), ([8, 16384, 5], 8), ([8, 300, 301, 302, 4], 3),
+])
+def test_partition_matches_oracle_bit_exact(dims, S):
+    from oracle import ist_oracle as O
+    w = _wl("p", dims, S, 4, 1, "fp32")
+    W, b, data = H.make_problem(w)
+    ctx, Wd, bd = H.gpu_context(w, W, b)
+    for seed in (0, 1, 2 ** 63 + 12345):
+        ctx.partition(seed)
+        gp = [tuple(t.cpu().numpy() for t in ctx.get_partition(l)) for l in range(1, ctx.t)]
+        ctx.reassemble()
+        ctx.sync_status()
+        _parts_equal(gp, O.partition(seed, dims, S))
+
+
+@pytest.mark.parametrize("precision", ["fp32", "bf16"])
+@pytest.mark.parametrize("dims,S", [([24, 100, 10], 3), ([16, 64, 72, 8], 4), ([8, 50, 41, 33, 6], 5)])
+def test_gathered_slices_are_the_oracles_slices_bit_exact(dims, S, precision):
+    from oracle import ist_oracle as O
+    w = _wl("g", dims, S, 4, 1, precision)
+    W, b, data = H.make_problem(w)
+    ctx, Wd, bd = H.gpu_context(w, W, b)
+    ctx.partition(9)
+    parts = O.partition(9, dims, S)
+    for s in range(S):
+        Ws, bs = O.slice_subnet(W, b, parts, s)
+        for l in range(1, ctx.t + 1):
+            gw, gb = ctx.get_subnet_params(l, s)
+            assert np.array_equal(gw.cpu().numpy(), Ws[l - 1])
+            assert np.array_equal(gb.cpu().numpy(), bs[l - 1])
+    ctx.reassemble()
+    ctx.sync_status()
+
+
+@pytest.mark.parametrize("precision", ["fp32", "bf16"])
+@pytest.mark.parametrize("dims,S", [([24, 100, 10], 3), ([16, 64, 72, 8], 4), ([1024, 4096, 4096, 35], 4)])
+def test_untouched_round_returns_the_network_bit_exact(dims, S, precision):
+    w = _wl("u", dims, S, 4, 1, precision)
+    W, b, data = H.make_problem(w)
+    ctx, Wd, bd = H.gpu_context(w, W, b)
+    for seed in (3, 4):
+        ctx.partition(seed)
+        ctx.reassemble()
+    ctx.sync_status()
+    for l in range(ctx.t):
+        assert np.array_equal(Wd[l].cpu().numpy(), W[l])
+        assert np.array_equal(bd[l].cpu().numpy(), b[l])
+
+
+# ---------------------------------------------------------------------------------------------
+# one full round
+# ---------------------------------------------------------------------------------------------
+
+def _check_round(w, rtol_w, rtol_dw, loss_tol, loss_rel, as_bf16=None, bias_scale=0.1):
+    W, b, data = H.make_problem(w, bias_scale=bias_scale)
+    seed = 4242
+    o, oparts, oloss = H.oracle_round(w, W, b, data, seed)
+    ctx, gW, gb, gparts, gloss = H.gpu_round(w, W, b, data, seed, as_bf16=as_bf16)
+    _parts_equal(gparts, oparts)
+    assert gloss.shape == oloss.shape
+    if loss_rel:
+        np.testing.assert_allclose(gloss, oloss, rtol=loss_tol, atol=0)
+    else:
+        assert abs(gloss.mean() - oloss.mean()) <= loss_tol, (gloss.mean(), oloss.mean())
+        assert np.max(np.abs(gloss - oloss)) <= 20 * loss_tol
+    for l in range(len(W)):
+        H.assert_close(gW[l], o.W[l], rtol_w, f"W_{l + 1}")
+        H.assert_close(gb[l], o.b[l], rtol_w, f"b_{l + 1}")
+        dg, do = gW[l].astype(np.float64) - W[l], o.W[l] - W[l]
+        fro = np.linalg.norm(dg - do) / max(np.linalg.norm(do), 1e-300)
+        assert fro <= rtol_dw, f"update of W_{l + 1}: {fro:.3e} > {rtol_dw}"
+        dbg, dbo = gb[l].astype(np.float64) - b[l], o.b[l] - b[l]
+        fro = np.linalg.norm(dbg - dbo) / max(np.linalg.norm(dbo), 1e-300)
+        assert fro <= rtol_dw, f"update of b_{l + 1}: {fro:.3e} > {rtol_dw}"
+    # entries of middle layers outside every subnet are bit-identical to the input
+    from oracle import ist_oracle as O
+    for l in range(2, len(W)):
+        g_prev = np.empty(w.layer_dims[l - 1], dtype=int)
+        g_cur = np.empty(w.layer_dims[l], dtype=int)
+        for s in range(w.S):
+            g_prev[O.group(oparts, l - 1, s)] = s
+            g_cur[O.group(oparts, l, s)] = s
+        cross = g_prev[:, None] != g_cur[None, :]
+        assert np.array_equal(gW[l - 1][cross], W[l - 1][cross])
+    return ctx
+
+
+def test_fp32_round_tiny_config():
+    # the 784 -> 1024 -> 10, S = 2, batch 128, K = 10 workload at full size
+    _check_round(synth.C1, FP32_RTOL, 1e-3, FP32_RTOL, True)
+
+
+@pytest.mark.parametrize("dims,S,B,K", [
+    ([20, 37, 5], 3, 7, 3),              # nothing divides anything
+    ([16, 64, 72, 8], 4, 16, 4),
+    ([33, 129, 65, 130, 11], 2, 33, 2),  # three hidden layers, ragged
+    ([12, 6], 1, 5, 3),                  # no hidden layer
+    ([9, 40, 4], 1, 1, 2),               # S = 1, batch 1
+    ([64, 256, 256, 35], 4, 64, 5),
+])
+def test_fp32_round_shapes(dims, S, B, K):
+    _check_round(_wl("s", dims, S, B, K, "fp32", lr=0.05), FP32_RTOL, 1e-3, FP32_RTOL, True)
+
+
+@pytest.mark.parametrize("dims,S,B,K,x_dist", [
+    ([1024, 4096, 4096, 35], 4, 256, 3, "normal"),         # speech-like shape, fewer steps
+    ([256, 1024, 1024, 35], 4, 256, 10, "normal"),
+    ([3072, 2048, 2048, 10], 8, 512, 2, "uniform_std"),   # wide-pixel shape at 1/8 width
+    ([24, 100, 10], 3, 19, 3, "normal"),                   # ragged everything
+    ([40, 72, 136, 200, 12], 2, 40, 2, "normal"),
+    ([1024, 2048, 2048, 100], 16, 512, 2, "normal"),       # sweep shape
+])
+def test_bf16_round_shapes(dims, S, B, K, x_dist):
+    _check_round(_wl("b", dims, S, B, K, "bf16", x_dist=x_dist), BF16_W_RTOL, BF16_DW_RTOL,
+                 BF16_LOSS_ATOL, False)
+
+
+def test_bf16_round_accepts_fp32_rows():
+    w = _wl("b32", [100, 64, 48, 7], 2, 24, 3, "bf16")
+    _check_round(w, BF16_W_RTOL, BF16_DW_RTOL, BF16_LOSS_ATOL, False, as_bf16=False)
+
+
+@pytest.mark.parametrize("precision", ["fp32", "bf16"])
+def test_csr_round(precision):
+    w = synth.Workload("csr", (5000, 256, 1000), S=4, B=32, K=3, rounds=1, precision=precision,
+                       x_dist="csr", lr=0.02, seed=5, csr_mean_nnz=20.0)
+    if precision == "fp32":
+        _check_round(w, FP32_RTOL, 1e-3, FP32_RTOL, True)
+    else:
+        _check_round(w, BF16_W_RTOL, BF16_DW_RTOL, BF16_LOSS_ATOL, False)
+
+
+def test_strides_zero_reuse_the_same_rows():
+    # stride_step = 0 and stride_subnet = 0: every subnet and step sees batch 0
+    import torch
+    from oracle import ist_oracle as O
+    w = _wl("z", [16, 32, 6], 2, 8, 3, "fp32", lr=0.05)
+    W, b, data = H.make_problem(w)
+    ctx, Wd, bd = H.gpu_context(w, W, b)
+    X, y = H.gpu_inputs(w, data)
+    ctx.partition(1)
+    gl = ctx.local_steps(X, y, w.lr, w.K, w.B, stride_subnet=0, stride_step=0).cpu().numpy()
+    ctx.reassemble()
+    ctx.sync_status()
+    Xr = np.broadcast_to(data.X[0, 0], data.X.shape).copy()
+    yr = np.broadcast_to(data.y[0, 0], data.y.shape).copy()
+    o = O.IstOracle(w.layer_dims, w.S)
+    o.bind_weights(W, b)
+    ol = o.round(1, Xr, yr, w.lr, w.K)
+    np.testing.assert_allclose(gl, ol, rtol=1e-4)
+    for l in range(2):
+        H.assert_close(Wd[l].cpu().numpy(), o.W[l], FP32_RTOL)
+
+
+def test_two_rounds_in_a_row_resample():
+    from oracle import ist_oracle as O
+    w = _wl("r", [32, 96, 80, 9], 4, 16, 3, "fp32", lr=0.05)
+    W, b, _ = H.make_problem(w)
+    ctx, Wd, bd = H.gpu_context(w, W, b)
+    o = O.IstOracle(w.layer_dims, w.S)
+    o.bind_weights(W, b)
+    for r in range(3):
+        data = synth.make_round_inputs(w, r)
+        X, y = H.gpu_inputs(w, data)
+        gl = ctx.round(100 + r, X, y, w.lr, w.K, w.B).cpu().numpy()
+        ol = o.round(100 + r, data.X, data.y, w.lr, w.K)
+        np.testing.assert_allclose(gl, ol, rtol=2e-4)
+    ctx.sync_status()
+    for l in range(3):
+        H.assert_close(Wd[l].cpu().numpy(), o.W[l], 3e-4)
+        H.assert_close(bd[l].cpu().numpy(), o.b[l], 3e-4)
+
+
+# ---------------------------------------------------------------------------------------------
+# eval
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dims,n,B", [([20, 37, 5], 50, 16), ([64, 128, 96, 10], 300, 128)])
+def test_eval_matches_oracle(dims, n, B):
+    import torch
+    from oracle import ist_oracle as O
+    w = _wl("e", dims, 1, B, 1, "fp32")
+    W, b, _ = H.make_problem(w, bias_scale=0.2)
+    X = synth.make_dense_inputs(1, 1, n, dims[0], "normal", 5)[0, 0]
+    y = synth.make_labels((n,), dims[-1], 5)
+    ctx, Wd, bd = H.gpu_context(w, W, b)
+    loss, correct = ctx.eval(torch.tensor(X, device="cuda:0"), torch.tensor(y, device="cuda:0"), n)
+    ctx.sync_status()
+    W64 = [x.astype(np.float64) for x in W]
+    b64 = [x.astype(np.float64) for x in b]
+    ol, oc = O.evaluate(W64, b64, X.astype(np.float64), y)
+    assert abs(loss.item() - ol) <= 1e-4 * abs(ol)
+    # the arg-max is decided in fp32 on the device and fp64 in the oracle: rows whose top-two
+    # margin is below fp32 resolution may differ; count them and allow that many
+    z = O.forward(W64, b64, X.astype(np.float64))[0][-1]
+    top2 = np.sort(z, axis=1)[:, -2:]
+    unsure = int(((top2[:, 1] - top2[:, 0]) < 1e-4 * np.abs(top2[:, 1]).clip(1e-6)).sum())
+    assert abs(correct.item() - oc) <= unsure
+
+
+def test_eval_csr_matches_oracle():
+    import torch
+    from oracle import ist_oracle as O
+    dims, n = (3000, 130, 50), 40
+    w = synth.Workload("ec", dims, S=2, B=16, K=1, rounds=1, precision="fp32", x_dist="csr", seed=8)
+    W, b, _ = H.make_problem(w, bias_scale=0.2)
+    rp, col, val = synth.make_csr_inputs(n, dims[0], 30.0, 3)
+    y = synth.make_labels((n,), dims[-1], 3)
+    ctx, Wd, bd = H.gpu_context(w, W, b)
+    X = (torch.tensor(rp, dtype=torch.int32, device="cuda:0"), torch.tensor(col, device="cuda:0"),
+         torch.tensor(val, device="cuda:0"))
+    loss, correct = ctx.eval(X, torch.tensor(y, device="cuda:0"), n)
+    ctx.sync_status()
+    ol, oc = O.evaluate([x.astype(np.float64) for x in W], [x.astype(np.float64) for x in b],
+                        O.CsrRows(rp, col, val.astype(np.float64)), y)
+    assert abs(loss.item() - ol) <= 1e-4 * abs(ol)
+    assert abs(correct.item() - oc) <= 1
+
+
+# ---------------------------------------------------------------------------------------------
+# errors are reported, not faults
+# ---------------------------------------------------------------------------------------------
+
+def test_call_order_and_bad_arguments():
+    import torch
+    from paper_1910_02120_b200 import api
+    w = _wl("o", [16, 32, 6], 2, 8, 2, "fp32")
+    W, b, data = H.make_problem(w)
+    ctx = api.Ist(w.layer_dims, w.S, api.IST_FP32, w.B)
+    X, y = H.gpu_inputs(w, data)
+    with pytest.raises(api.IstError) as e:
+        ctx.partition(1)                       # nothing bound
+    assert e.value.status == api.IST_ERR_STATE
+    Wd = [torch.tensor(x, device="cuda:0") for x in W]
+    bd = [torch.tensor(x, device="cuda:0") for x in b]
+    ctx.bind_weights(Wd, bd)
+    with pytest.raises(api.IstError) as e:
+        ctx.local_steps(X, y, 0.1, 2, w.B)     # no partition
+    assert e.value.status == api.IST_ERR_STATE
+    ctx.partition(1)
+    with pytest.raises(api.IstError) as e:
+        ctx.partition(2)                       # partition already in place
+    assert e.value.status == api.IST_ERR_STATE
+    with pytest.raises(api.IstError) as e:
+        ctx.local_steps(X, y, 0.1, 2, w.B + 1)  # batch > max_batch
+    assert e.value.status == api.IST_ERR_ARG
+    with pytest.raises(api.IstError) as e:
+        ctx.local_steps(X, y, 0.1, 0, w.B)
+    assert e.value.status == api.IST_ERR_ARG
+    with pytest.raises(api.IstError) as e:
+        ctx.eval(X, y, 4)                      # eval while partitioned
+    assert e.value.status == api.IST_ERR_STATE
+    ctx.reassemble()
+    ctx.sync_status()
+
+
+def test_out_of_range_label_sets_the_device_status():
+    import torch
+    from paper_1910_02120_b200 import api
+    w = _wl("l", [16, 32, 6], 2, 8, 1, "fp32")
+    W, b, data = H.make_problem(w)
+    ctx, Wd, bd = H.gpu_context(w, W, b)
+    X, y = H.gpu_inputs(w, data)
+    y[3] = 6                                   # one past the last class
+    ctx.partition(1)
+    ctx.local_steps(X, y, 0.1, 1, w.B)
+    ctx.reassemble()
+    with pytest.raises(api.IstError) as e:
+        ctx.sync_status()
+    assert e.value.status == api.IST_ERR_DEVICE_CHECK
+    torch.cuda.synchronize()                   # the context is still usable
+    assert torch.isfinite(Wd[0]).all()
