@@ -254,10 +254,12 @@ ist_status check_input(ist_ctx* c, const ist_input* X, const int32_t* y, bool tr
 }
 
 // ---- grouped GEMM dispatch ------------------------------------------------------------------
-template <typename T>
-void gemm(ist_ctx* c, const GemmArgs<T>& a) {
-  gemm_simt<T>(c->launch(), a);
+// fp32 operands run on the CUDA cores, bf16 operands on the tensor cores.
+bool gemm(ist_ctx* c, const GemmArgs<float>& a) {
+  gemm_simt<float>(c->launch(), a);
+  return true;
 }
+bool gemm(ist_ctx* c, const GemmArgs<bf16>& a) { return gemm_tc(c->launch(), a, c->status()); }
 
 // One call of ist_local_steps in operand type T.
 template <typename T>
@@ -311,6 +313,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       }
       GemmArgs<T> g{};
       g.M = B; g.N = (int)c->np[l]; g.K = (int)c->np[l - 1]; g.G = S;
+      g.N_store = (int)c->ld[l];
       g.A = in_ptr(l - 1); g.a_sm = in_ld(l - 1); g.a_sk = 1; g.a_sg = in_sg(l - 1);
       g.B = weights(l); g.b_sn = 1; g.b_sk = c->ld[l]; g.b_sg = c->slice_elems(l);
       g.bias = c->bias(l); g.bias_sg = c->ld[l];
@@ -322,7 +325,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.outf = logits; g.outf_ld = c->ld[t]; g.outf_sg = Bm * c->ld[t];
       }
       Scope sc(c, IST_K_FWD);
-      gemm<T>(c, g);
+      if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "forward GEMM of layer %d cannot be launched", l);
     }
     // ---- loss and its gradient -------------------------------------------------------------
     {
@@ -336,13 +339,14 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       if (l > 1) {
         GemmArgs<T> g{};
         g.M = B; g.N = (int)c->np[l - 1]; g.K = (int)c->np[l]; g.G = S;
+        g.N_store = (int)c->ld[l - 1];
         g.A = delta(l); g.a_sm = c->ld[l]; g.a_sk = 1; g.a_sg = Bm * c->ld[l];
         g.B = weights(l); g.b_sn = c->ld[l]; g.b_sk = 1; g.b_sg = c->slice_elems(l);
         g.epi = EPI_RELU_MASK;
         g.mask = act(l - 1); g.mask_ld = c->ld[l - 1]; g.mask_sg = Bm * c->ld[l - 1];
         g.out = delta(l - 1); g.out_ld = c->ld[l - 1]; g.out_sg = Bm * c->ld[l - 1];
         Scope sc(c, IST_K_DX);
-        gemm<T>(c, g);
+        if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMM of layer %d cannot be launched", l);
       }
       {
         Scope sc(c, IST_K_BIAS_SGD);
@@ -357,6 +361,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       }
       GemmArgs<T> g{};
       g.M = (int)c->np[l - 1]; g.N = (int)c->np[l]; g.K = B; g.G = S;
+      g.N_store = (int)c->ld[l];
       g.A = in_ptr(l - 1); g.a_sm = 1; g.a_sk = in_ld(l - 1); g.a_sg = in_sg(l - 1);
       g.B = delta(l); g.b_sn = 1; g.b_sk = c->ld[l]; g.b_sg = Bm * c->ld[l];
       g.epi = EPI_SGD;
@@ -364,7 +369,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       g.opw = c->opw(l);
       g.lr = lr;
       Scope sc(c, IST_K_DW_SGD);
-      gemm<T>(c, g);
+      if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "weight-gradient GEMM of layer %d cannot be launched", l);
     }
   }
   IST_CUDA(c, cudaGetLastError());

@@ -52,6 +52,7 @@ enum Epilogue : int {
 template <typename T>
 struct GemmArgs {
   int M, N, K, G;
+  int N_store;  // columns the epilogue may write (>= N, the padded row length); 0 = N
   const T* A; int64_t a_sm, a_sk, a_sg;
   const T* B; int64_t b_sn, b_sk, b_sg;
   int epi;
@@ -63,6 +64,9 @@ struct GemmArgs {
   float lr;
 };
 template <typename T> void gemm_simt(const Launch& L, const GemmArgs<T>& a);
+// Tensor-core path (tcgen05 + TMA) for bf16 operands.  Returns false if the shape cannot be
+// described to TMA (misaligned strides) or the operand layouts do not fit an epilogue.
+bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st);
 
 // ---- rowops.cu --------------------------------------------------------------------------
 // Row-wise softmax cross-entropy of logits [G][B][ld] against labels; writes
