@@ -40,6 +40,10 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C3", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--local-steps", type=int, default=0,
+                    help="override K (local steps per round); makes a small case for profiler captures")
+    ap.add_argument("--quick", action="store_true",
+                    help="device-timed pass only (no end-to-end, per-class or CPU passes), warm-up as given")
     return ap.parse_args()
 
 
@@ -286,7 +290,8 @@ def run_ours(args, w):
         return ms
 
     # ---- device-resident timing ---------------------------------------------------------------
-    for i in range(max(args.warmup, 3)):
+    n_warm = args.warmup if args.quick else max(args.warmup, 3)
+    for i in range(n_warm):
         one_round(i, X_of(dev_in), y_dev)
     ctx.sync_status()
     sampler = ClockSampler(local)
@@ -304,6 +309,14 @@ def run_ours(args, w):
     ms = max_over_ranks(e0.elapsed_time(e1))
     ctx.sync_status()
     value = world * w.samples_per_round * args.steps / (ms * 1e-3)
+    if args.quick:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                              "warmup": n_warm, "ms_per_step": ms / args.steps, "quick": True,
+                              "gpu_launches": launches, "config": config_dict(w, world)}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- end to end: host buffers in, loss out, copies inside the timed region ------------------
     stage_in = [torch.empty_like(t, device=dev) for t in host_in]
@@ -386,7 +399,7 @@ def run_ours(args, w):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "warmup": n_warm, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.precision.replace("fp", "f"), "data": "synthetic",
         "config": config_dict(w, world), "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -401,6 +414,8 @@ def run_ours(args, w):
 def main():
     args = parse_args()
     w = synth.WORKLOADS[args.config]
+    if args.local_steps > 0:
+        w = w.scaled(K=args.local_steps, name=w.name + f"-K{args.local_steps}")
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -1,28 +1,33 @@
 // Grouped bf16 GEMM on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
 // memory, operands staged in shared memory by TMA) with the local-step epilogues fused in:
 // bias + ReLU (forward), logits, ReLU mask (delta back-propagation) and the SGD update of the
-// fp32 master slice with its bf16 operand copy (paper Sec. 2.1 "Training Subnets"; App. A
-// Eq. (2) on the slices).  All S subnets run as the third grid dimension of one launch.
+// fp32 master slice together with its bf16 operand copy (paper Sec. 2.1 "Training Subnets";
+// App. A Eq. (2) on the slices).  All S subnets are tiles of one persistent launch.
 //
 //   C[g](m, n) = sum_k A[g](m, k) * B[g](n, k),   fp32 accumulation
 //
-// One CTA computes one 128 x BN tile.  Warp 0 (one lane) issues TMA loads into a ring of
-// STAGES shared-memory slots; warp 1 (one lane) issues the MMAs and owns the tensor-memory
-// allocation; warps 2..5 read the accumulator back (tcgen05.ld: warp w may touch lanes
-// 32*(w%4)..+31) and apply the epilogue straight from registers.
+// One CTA per SM walks over 128 x BN output tiles (tile = blockIdx.x + i * gridDim.x).
+//   warp 0 (one lane)  TMA loads of the A / B k-slabs into a ring of STAGES slots
+//   warp 1 (one lane)  tcgen05.mma issue; owns the tensor-memory allocation (2 accumulators,
+//                      so the MMAs of tile i+1 overlap the epilogue of tile i)
+//   warps 2..5         epilogue: tcgen05.ld (warp w reads lanes 32*(w%4)..+31, one row per
+//                      thread), 32 columns at a time, staged in swizzled shared memory and
+//                      written with TMA stores (coalesced, clipped at the tensor edge)
+//   warp 6 (one lane)  TMA loads of the epilogue's input chunks: the fp32 master slice for the
+//                      SGD update, the ReLU mask for the delta GEMM
+// The weight-update epilogue is the HBM-heavy part of a step (10 bytes per weight against
+// 2*B flops): its master chunks are prefetched up to four chunks ahead while earlier chunks are
+// updated in place in shared memory and stored back.
 //
-// Either operand may be contiguous along k ("K-major": activations in x*W, weights in
-// delta*W^T) or along m/n ("MN-major": weights in x*W, both operands of a^T*delta); the shared
-// memory tile is 128-byte swizzled in both cases and the UMMA descriptors say which.
-// Rows/columns beyond the tensor extents are zero-filled by TMA, so ragged shapes need no
-// special casing in the main loop; the epilogue masks its stores.
+// Either operand may be contiguous along k ("K-major") or along m/n ("MN-major"); the shared
+// memory tile is 128-byte swizzled in both cases and the UMMA descriptors say which.  Rows and
+// columns beyond the tensor extents are zero-filled by TMA loads and dropped by TMA stores.
 //
 // Every wait is bounded: after about a second without progress a role records
 // IST_ERR_DEVICE_TIMEOUT in the status word, raises the CTA's abort flag and all roles fall
 // through to the common exit, where tensor memory is released.
 #include <cuda.h>
 
-#include <cstdio>
 #include <map>
 #include <mutex>
 #include <tuple>
@@ -34,7 +39,9 @@ namespace {
 
 constexpr int BM = 128;
 constexpr int BK = 64;                   // 64 bf16 = 128 bytes = one swizzle row
-constexpr int kThreads = 192;
+constexpr int CH = 32;                   // epilogue chunk: 32 output columns
+constexpr int kThreads = 224;
+constexpr int kEpiThreads = 128;
 constexpr long long kWaitLimitCycles = 2000000000ll;   // ~1 s at 2 GHz
 
 // ---- small PTX wrappers ------------------------------------------------------------------------
@@ -47,6 +54,9 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
@@ -81,6 +91,33 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+__device__ __forceinline__ void tma_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+// AND-reduction of a predicate over the epilogue threads, so that all of them leave together
+// when a bounded wait has expired for any of them.
+__device__ __forceinline__ bool epi_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 p, %1, 0;\n\t"
+      "bar.red.and.pred q, 2, %2, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)ok), "n"(kEpiThreads)
+      : "memory");
+  return r != 0;
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -133,90 +170,95 @@ __host__ __device__ constexpr uint32_t make_idesc(int a_mn, int b_mn, int n) {
 }
 
 struct TcArgs {
-  int M, N, K;            // M, N: bounds of the output rows / columns the epilogue may touch
+  int M, N, K;            // M, N: bounds of the output rows / columns the epilogue touches
+  int m_tiles, n_tiles, G;
   int a_gmul, b_gmul;     // 1 if the operand has one slab per group, 0 if all groups share it
-  int epi;
   const float* bias; long long bias_sg;
-  bf16* out; long long out_ld, out_sg;
-  float* outf; long long outf_ld, outf_sg;
-  const bf16* mask; long long mask_ld, mask_sg;
-  bf16* opw;
   float lr;
   DeviceStatus* status;
 };
 
-__device__ __forceinline__ uint2 pack4(float a, float b, float c, float d) {
-  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-  uint2 r;
-  r.x = *reinterpret_cast<uint32_t*>(&lo);
-  r.y = *reinterpret_cast<uint32_t*>(&hi);
+// What each epilogue keeps in a chunk slot: an fp32 area ([128][32] floats, 128-byte swizzle)
+// and / or a bf16 area ([128][32] bf16, 64-byte swizzle); whether a chunk is loaded before use.
+template <int EPI> struct EpiTraits;
+template <> struct EpiTraits<EPI_BIAS_RELU> { static constexpr bool k32 = false, k16 = true, kAux = false; };
+template <> struct EpiTraits<EPI_BIAS_F32> { static constexpr bool k32 = true, k16 = false, kAux = false; };
+template <> struct EpiTraits<EPI_RELU_MASK> { static constexpr bool k32 = false, k16 = true, kAux = true; };
+template <> struct EpiTraits<EPI_SGD> { static constexpr bool k32 = true, k16 = true, kAux = true; };
+
+__device__ __forceinline__ uint4 pack8(const float* v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
+  uint4 r;
+  r.x = *reinterpret_cast<uint32_t*>(&a);
+  r.y = *reinterpret_cast<uint32_t*>(&b);
+  r.z = *reinterpret_cast<uint32_t*>(&c);
+  r.w = *reinterpret_cast<uint32_t*>(&d);
   return r;
 }
-
-// Applies the epilogue to 32 consecutive columns [n, n+32) of output row m (thread-private).
-template <int EPI>
-__device__ __forceinline__ void epilogue_row32(const TcArgs& a, int g, int m, int n, const uint32_t* acc) {
-#pragma unroll
-  for (int v = 0; v < 8; ++v) {
-    const int nn = n + 4 * v;
-    if (nn >= a.N) break;
-    float c0 = __uint_as_float(acc[4 * v]), c1 = __uint_as_float(acc[4 * v + 1]);
-    float c2 = __uint_as_float(acc[4 * v + 2]), c3 = __uint_as_float(acc[4 * v + 3]);
-    if (EPI == EPI_BIAS_RELU) {
-      float4 b = *reinterpret_cast<const float4*>(a.bias + (long long)g * a.bias_sg + nn);
-      *reinterpret_cast<uint2*>(a.out + (long long)g * a.out_sg + (long long)m * a.out_ld + nn) =
-          pack4(fmaxf(c0 + b.x, 0.f), fmaxf(c1 + b.y, 0.f), fmaxf(c2 + b.z, 0.f), fmaxf(c3 + b.w, 0.f));
-    } else if (EPI == EPI_BIAS_F32) {
-      float4 b = *reinterpret_cast<const float4*>(a.bias + (long long)g * a.bias_sg + nn);
-      *reinterpret_cast<float4*>(a.outf + (long long)g * a.outf_sg + (long long)m * a.outf_ld + nn) =
-          make_float4(c0 + b.x, c1 + b.y, c2 + b.z, c3 + b.w);
-    } else if (EPI == EPI_RELU_MASK) {
-      uint2 mk = *reinterpret_cast<const uint2*>(a.mask + (long long)g * a.mask_sg + (long long)m * a.mask_ld + nn);
-      __nv_bfloat162 m01 = *reinterpret_cast<__nv_bfloat162*>(&mk.x);
-      __nv_bfloat162 m23 = *reinterpret_cast<__nv_bfloat162*>(&mk.y);
-      *reinterpret_cast<uint2*>(a.out + (long long)g * a.out_sg + (long long)m * a.out_ld + nn) =
-          pack4(__low2float(m01) > 0.f ? c0 : 0.f, __high2float(m01) > 0.f ? c1 : 0.f,
-                __low2float(m23) > 0.f ? c2 : 0.f, __high2float(m23) > 0.f ? c3 : 0.f);
-    } else if (EPI == EPI_SGD) {
-      long long o = (long long)g * a.outf_sg + (long long)m * a.outf_ld + nn;
-      float4 w = *reinterpret_cast<float4*>(a.outf + o);
-      w.x -= a.lr * c0; w.y -= a.lr * c1; w.z -= a.lr * c2; w.w -= a.lr * c3;
-      *reinterpret_cast<float4*>(a.outf + o) = w;
-      *reinterpret_cast<uint2*>(a.opw + o) = pack4(w.x, w.y, w.z, w.w);
-    } else {
-      *reinterpret_cast<uint2*>(a.out + (long long)g * a.out_sg + (long long)m * a.out_ld + nn) =
-          pack4(c0, c1, c2, c3);
-    }
-  }
+__device__ __forceinline__ void unpack8(uint4 u, float* v) {
+  __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&u.x), b = *reinterpret_cast<__nv_bfloat162*>(&u.y);
+  __nv_bfloat162 c = *reinterpret_cast<__nv_bfloat162*>(&u.z), d = *reinterpret_cast<__nv_bfloat162*>(&u.w);
+  v[0] = __low2float(a); v[1] = __high2float(a); v[2] = __low2float(b); v[3] = __high2float(b);
+  v[4] = __low2float(c); v[5] = __high2float(c); v[6] = __low2float(d); v[7] = __high2float(d);
 }
 
-template <int A_MN, int B_MN, int BN, int STAGES, int EPI>
-__global__ void __launch_bounds__(kThreads)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcArgs a) {
+// Row r of a chunk slot.  fp32 area: 128-byte rows, 16-byte unit u stored at u ^ (r & 7).
+// bf16 area: 64-byte rows, 16-byte unit u stored at u ^ ((r >> 1) & 3).
+__device__ __forceinline__ float4* f32_unit(uint8_t* area, int r, int u) {
+  return reinterpret_cast<float4*>(area + r * 128 + ((u ^ (r & 7)) << 4));
+}
+__device__ __forceinline__ uint4* b16_unit(uint8_t* area, int r, int u) {
+  return reinterpret_cast<uint4*>(area + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
+}
+
+template <int A_MN, int B_MN, int BN, int STAGES, int SLOTS, int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmC32,   // fp32 chunks: logits out, master in/out
+               const __grid_constant__ CUtensorMap tmC16,   // bf16 chunks out: activations, delta, weights
+               const __grid_constant__ CUtensorMap tmAux16, // bf16 chunks in: ReLU mask
+               TcArgs a) {
+  using ET = EpiTraits<EPI>;
   constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr uint32_t F32_BYTES = ET::k32 ? BM * CH * 4 : 0, B16_BYTES = ET::k16 ? BM * CH * 2 : 0;
+  constexpr uint32_t SLOT_BYTES = F32_BYTES + B16_BYTES;
+  constexpr uint32_t AUX_BYTES = EPI == EPI_SGD ? F32_BYTES : B16_BYTES;
+  constexpr uint32_t TMEM_COLS = 2 * BN;
+  constexpr int NCH = BN / CH;
+
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
+  uint8_t* slots = smem + STAGES * STAGE_BYTES;
+  __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
+  __shared__ uint64_t slot_full[SLOTS], slot_empty[SLOTS];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, g = blockIdx.z;
   const int num_kb = (a.K + BK - 1) / BK;
+  const int total_tiles = a.m_tiles * a.n_tiles * a.G;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(&acc_bar, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 4);      // one arrival per epilogue warp
+    }
+    for (int s = 0; s < SLOTS; ++s) {
+      mbar_init(&slot_full[s], 1);
+      mbar_init(&slot_empty[s], 1);
+    }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    fence_async_smem();
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
-                 "r"((uint32_t)BN)
+                 "r"(TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -227,73 +269,204 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   volatile int* abortp = &abort_flag;
 
   if (warp == 0) {
+    // ---------------------------------------------------------------- operand loads
     if (lane == 0) {
-      int issued = 0;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(&empty_bar[s], ph ^ 1, abortp, a.status, 1)) break;
-        uint8_t* sa = smem + s * STAGE_BYTES;
-        uint8_t* sb = sa + A_BYTES;
-        mbar_expect_tx(&full_bar[s], STAGE_BYTES);
-        if (A_MN) {
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % a.m_tiles) * BM;
+        const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
+        const int g = tile / (a.m_tiles * a.n_tiles);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          ok = mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abortp, a.status, 1);
+          if (!ok) break;
+          uint8_t* sa = smem + s * STAGE_BYTES;
+          uint8_t* sb = sa + A_BYTES;
+          mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+          if (A_MN) {
 #pragma unroll
-          for (int j = 0; j < BM / 64; ++j)
-            tma_load_3d(sa + j * (BK * 128), &tmA, &full_bar[s], m0 + 64 * j, kb * BK, g * a.a_gmul);
-        } else {
-          tma_load_3d(sa, &tmA, &full_bar[s], kb * BK, m0, g * a.a_gmul);
-        }
-        if (B_MN) {
+            for (int j = 0; j < BM / 64; ++j)
+              tma_load_3d(sa + j * (BK * 128), &tmA, &full_bar[s], m0 + 64 * j, kb * BK, g * a.a_gmul);
+          } else {
+            tma_load_3d(sa, &tmA, &full_bar[s], kb * BK, m0, g * a.a_gmul);
+          }
+          if (B_MN) {
 #pragma unroll
-          for (int j = 0; j < BN / 64; ++j)
-            tma_load_3d(sb + j * (BK * 128), &tmB, &full_bar[s], n0 + 64 * j, kb * BK, g * a.b_gmul);
-        } else {
-          tma_load_3d(sb, &tmB, &full_bar[s], kb * BK, n0, g * a.b_gmul);
+            for (int j = 0; j < BN / 64; ++j)
+              tma_load_3d(sb + j * (BK * 128), &tmB, &full_bar[s], n0 + 64 * j, kb * BK, g * a.b_gmul);
+          } else {
+            tma_load_3d(sb, &tmB, &full_bar[s], kb * BK, n0, g * a.b_gmul);
+          }
         }
-        issued = kb + 1;
       }
-      if (*abortp) {
+      if (!ok) {
         // let copies already in flight land before the CTA's shared memory goes away
-        for (int kb = max(0, issued - STAGES); kb < issued; ++kb) {
+        for (int j = max(0, it - STAGES); j < it; ++j) {
           long long t0 = clock64();
-          while (!mbar_try_wait(&full_bar[kb % STAGES], (kb / STAGES) & 1) && clock64() - t0 < kWaitLimitCycles) {}
+          while (!mbar_try_wait(&full_bar[j % STAGES], (j / STAGES) & 1) && clock64() - t0 < kWaitLimitCycles) {}
         }
       }
     }
   } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issue
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BN);
+      int it = 0, j = 0;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        ok = mbar_wait(&full_bar[s], ph, abortp, a.status, 2);
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++j) {
+        const int b = j & 1;
+        ok = mbar_wait(&acc_empty[b], ((j >> 1) & 1) ^ 1, abortp, a.status, 2);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
+        const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          ok = mbar_wait(&full_bar[s], (it / STAGES) & 1, abortp, a.status, 3);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
 #pragma unroll
-        for (int k = 0; k < BK / 16; ++k) {
-          // K-major: 16 k-elements = 32 bytes inside the swizzle row; 8-row groups 1024 B apart.
-          // MN-major: 16 k-rows = 2048 B; 64-element MN chunks (one TMA box each) 8192 B apart.
-          const uint64_t ad = A_MN ? make_desc(sa + k * 2048, BK * 128, 1024) : make_desc(sa + k * 32, 16, 1024);
-          const uint64_t bd = B_MN ? make_desc(sb + k * 2048, BK * 128, 1024) : make_desc(sb + k * 32, 16, 1024);
-          tc_mma(tmem_base, ad, bd, idesc, (kb | k) != 0);
+          for (int k = 0; k < BK / 16; ++k) {
+            // K-major: 16 k-elements = 32 bytes inside the swizzle row; 8-row groups 1024 B apart.
+            // MN-major: 16 k-rows = 2048 B; 64-element MN chunks (one TMA box each) 8192 B apart.
+            const uint64_t ad = A_MN ? make_desc(sa + k * 2048, BK * 128, 1024) : make_desc(sa + k * 32, 16, 1024);
+            const uint64_t bd = B_MN ? make_desc(sb + k * 2048, BK * 128, 1024) : make_desc(sb + k * 32, 16, 1024);
+            tc_mma(d_tmem, ad, bd, idesc, (kb | k) != 0);
+          }
+          tc_commit(&empty_bar[s]);   // frees the slot once these MMAs have read it
         }
-        tc_commit(&empty_bar[s]);   // frees the slot once these MMAs have read it
+        if (ok) tc_commit(&acc_full[b]);
       }
-      if (ok) tc_commit(&acc_bar);  // accumulator complete
     }
-  } else {
-    if (mbar_wait(&acc_bar, 0, abortp, a.status, 3)) {
+  } else if (warp < 6) {
+    // ---------------------------------------------------------------- epilogue
+    const int q = warp & 3;
+    const int r = q * 32 + lane;                      // row of the tile owned by this thread
+    const bool leader = threadIdx.x == 64;            // issues the TMA stores
+    int cq = 0, j = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++j) {
+      const int m0 = (tile % a.m_tiles) * BM;
+      const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
+      const int g = tile / (a.m_tiles * a.n_tiles);
+      const int b = j & 1;
+      ok = epi_all(mbar_wait(&acc_full[b], (j >> 1) & 1, abortp, a.status, 4));
+      if (!ok) break;
       tc_fence_after();
-      const int q = warp & 3;
-      const int m = m0 + q * 32 + lane;
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
-        if (n0 + c >= a.N) break;   // warp-uniform
+      for (int c = 0; c < NCH; ++c, ++cq) {
+        const int nc = n0 + c * CH;
+        if (nc >= a.N) break;                         // CTA-uniform
+        const int slot = cq % SLOTS;
+        uint8_t* f32 = slots + slot * SLOT_BYTES;
+        uint8_t* b16 = f32 + F32_BYTES;
+        if (ET::kAux) {
+          ok = epi_all(mbar_wait(&slot_full[slot], (cq / SLOTS) & 1, abortp, a.status, 5));
+          if (!ok) break;
+        }
         uint32_t acc[32];
-        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c, acc);
-        if (m < a.M) epilogue_row32<EPI>(a, g, m, n0 + c, acc);
+        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * CH), acc);
+        if (EPI == EPI_SGD) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {               // 8 columns per iteration
+            float w[8];
+            float4 w0 = *f32_unit(f32, r, 2 * u), w1 = *f32_unit(f32, r, 2 * u + 1);
+            w[0] = w0.x - a.lr * __uint_as_float(acc[8 * u + 0]);
+            w[1] = w0.y - a.lr * __uint_as_float(acc[8 * u + 1]);
+            w[2] = w0.z - a.lr * __uint_as_float(acc[8 * u + 2]);
+            w[3] = w0.w - a.lr * __uint_as_float(acc[8 * u + 3]);
+            w[4] = w1.x - a.lr * __uint_as_float(acc[8 * u + 4]);
+            w[5] = w1.y - a.lr * __uint_as_float(acc[8 * u + 5]);
+            w[6] = w1.z - a.lr * __uint_as_float(acc[8 * u + 6]);
+            w[7] = w1.w - a.lr * __uint_as_float(acc[8 * u + 7]);
+            *f32_unit(f32, r, 2 * u) = make_float4(w[0], w[1], w[2], w[3]);
+            *f32_unit(f32, r, 2 * u + 1) = make_float4(w[4], w[5], w[6], w[7]);
+            *b16_unit(b16, r, u) = pack8(w);
+          }
+        } else if (EPI == EPI_RELU_MASK) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            float mk[8], o[8];
+            unpack8(*b16_unit(b16, r, u), mk);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o[e] = mk[e] > 0.f ? __uint_as_float(acc[8 * u + e]) : 0.f;
+            *b16_unit(b16, r, u) = pack8(o);
+          }
+        } else {
+          const float* bias = a.bias + (long long)g * a.bias_sg;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            float o[8];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int n = nc + 8 * u + 4 * h;
+              float4 bv = n < a.N ? __ldg(reinterpret_cast<const float4*>(bias + n)) : make_float4(0.f, 0.f, 0.f, 0.f);
+              o[4 * h + 0] = __uint_as_float(acc[8 * u + 4 * h + 0]) + bv.x;
+              o[4 * h + 1] = __uint_as_float(acc[8 * u + 4 * h + 1]) + bv.y;
+              o[4 * h + 2] = __uint_as_float(acc[8 * u + 4 * h + 2]) + bv.z;
+              o[4 * h + 3] = __uint_as_float(acc[8 * u + 4 * h + 3]) + bv.w;
+            }
+            if (EPI == EPI_BIAS_RELU) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) o[e] = fmaxf(o[e], 0.f);
+              *b16_unit(b16, r, u) = pack8(o);
+            } else {
+              *f32_unit(f32, r, 2 * u) = make_float4(o[0], o[1], o[2], o[3]);
+              *f32_unit(f32, r, 2 * u + 1) = make_float4(o[4], o[5], o[6], o[7]);
+            }
+          }
+        }
+        fence_async_smem();          // generic-proxy writes -> visible to the TMA store
+        epi_barrier();
+        if (leader) {
+          if (ET::k32) tma_store_3d(&tmC32, f32, nc, m0, g);
+          if (ET::k16) tma_store_3d(&tmC16, b16, nc, m0, g);
+          tma_commit_group();
+          if (ET::kAux) {
+            // the slot of the previous chunk may be refilled once its store has read it
+            tma_wait_read<1>();
+            if (cq >= 1) mbar_arrive(&slot_empty[(cq - 1) % SLOTS]);
+          } else {
+            // no loader: this thread alone gates slot reuse.  The others run at most one chunk
+            // ahead of it (they meet it again at the next barrier), so all but the newest
+            // SLOTS - 2 stores must have read their slots before it goes on.
+            tma_wait_read<(SLOTS >= 2 ? SLOTS - 2 : 0)>();
+          }
+        }
+      }
+      if (!ok) break;
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[b]);
+    }
+    if (leader) tma_wait_all();      // all stores complete before the CTA exits
+  } else {
+    // ---------------------------------------------------------------- epilogue input loads
+    if (ET::kAux && lane == 0) {
+      int cq = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % a.m_tiles) * BM;
+        const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
+        const int g = tile / (a.m_tiles * a.n_tiles);
+        for (int c = 0; c < NCH; ++c, ++cq) {
+          const int nc = n0 + c * CH;
+          if (nc >= a.N) break;
+          const int slot = cq % SLOTS;
+          ok = mbar_wait(&slot_empty[slot], ((cq / SLOTS) & 1) ^ 1, abortp, a.status, 6);
+          if (!ok) break;
+          uint8_t* f32 = slots + slot * SLOT_BYTES;
+          mbar_expect_tx(&slot_full[slot], AUX_BYTES);
+          if (EPI == EPI_SGD) tma_load_3d(f32, &tmC32, &slot_full[slot], nc, m0, g);
+          else tma_load_3d(f32 + F32_BYTES, &tmAux16, &slot_full[slot], nc, m0, g);
+        }
+      }
+      if (!ok) {
+        for (int jq = max(0, cq - SLOTS); jq < cq; ++jq) {
+          long long t0 = clock64();
+          while (!mbar_try_wait(&slot_full[jq % SLOTS], (jq / SLOTS) & 1) && clock64() - t0 < kWaitLimitCycles) {}
+        }
       }
     }
   }
@@ -301,7 +474,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   if (warp == 1) {
     __syncwarp();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)BN)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
                  : "memory");
   }
 }
@@ -325,8 +498,20 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 tensor [groups][outer][inner] (inner contiguous), box {64, box_outer, 1}, 128-byte swizzle.
-using MapKey = std::tuple<const void*, long long, long long, long long, long long, long long, int>;
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+// Tensor [groups][outer][inner] (inner contiguous, strides in elements) with box
+// {box_inner, box_outer, 1}.  elem_bytes 2 = bf16, 4 = fp32.  swizzle_bytes 128 or 64.
+using MapKey = std::tuple<const void*, long long, long long, long long, long long, long long, int, int, int, int>;
 std::map<MapKey, CUtensorMap>& map_cache() {
   static std::map<MapKey, CUtensorMap> c;
   return c;
@@ -336,9 +521,11 @@ std::mutex& map_mutex() {
   return m;
 }
 
-bool make_map(CUtensorMap* out, const bf16* base, long long inner, long long outer, long long groups,
-              long long outer_stride, long long group_stride, int box_outer) {
-  MapKey key{base, inner, outer, groups, outer_stride, group_stride, box_outer};
+bool make_map(CUtensorMap* out, const void* base, int elem_bytes, long long inner, long long outer,
+              long long groups, long long outer_stride, long long group_stride, int box_inner, int box_outer,
+              int swizzle_bytes) {
+  if (!base) return false;
+  MapKey key{base, inner, outer, groups, outer_stride, group_stride, elem_bytes, box_inner, box_outer, swizzle_bytes};
   std::lock_guard<std::mutex> lk(map_mutex());
   auto& cache = map_cache();
   auto it = cache.find(key);
@@ -349,54 +536,55 @@ bool make_map(CUtensorMap* out, const bf16* base, long long inner, long long out
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)groups};
-  cuuint64_t strides[2] = {(cuuint64_t)outer_stride * 2,
-                           (cuuint64_t)(groups > 1 ? group_stride : outer_stride * outer) * 2};
-  cuuint32_t box[3] = {64, (cuuint32_t)box_outer, 1};
+  cuuint64_t strides[2] = {(cuuint64_t)outer_stride * elem_bytes,
+                           (cuuint64_t)(groups > 1 ? group_stride : outer_stride * outer) * elem_bytes};
+  cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = fn(out, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
+                  const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   if (cache.size() > 4096) cache.clear();
   cache[key] = *out;
   return true;
 }
 
-template <int A_MN, int B_MN, int BN, int STAGES, int EPI>
-bool launch(const Launch& L, const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& t, int m_tiles, int n_tiles,
-            int G) {
-  constexpr int smem = STAGES * (BM * BK * 2 + BN * BK * 2) + 1024;
-  auto kern = gemm_tc_kernel<A_MN, B_MN, BN, STAGES, EPI>;
+struct Maps {
+  CUtensorMap a, b, c32, c16, aux16;
+};
+
+template <int A_MN, int B_MN, int BN, int STAGES, int SLOTS, int EPI>
+bool launch(const Launch& L, const Maps& m, const TcArgs& t) {
+  using ET = EpiTraits<EPI>;
+  constexpr int slot_bytes = (ET::k32 ? BM * CH * 4 : 0) + (ET::k16 ? BM * CH * 2 : 0);
+  constexpr int smem = STAGES * (BM * BK * 2 + BN * BK * 2) + SLOTS * slot_bytes + 1024;
+  static_assert(smem <= 227 * 1024 - 512, "shared memory budget exceeded");
+  auto kern = gemm_tc_kernel<A_MN, B_MN, BN, STAGES, SLOTS, EPI>;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
     configured = true;
   }
-  kern<<<dim3(m_tiles, n_tiles, G), kThreads, smem, L.stream>>>(ma, mb, t);
+  const int total = t.m_tiles * t.n_tiles * t.G;
+  const int grid = total < sm_count() ? total : sm_count();
+  kern<<<grid, kThreads, smem, L.stream>>>(m.a, m.b, m.c32, m.c16, m.aux16, t);
   L.count();
   return true;
 }
 
-template <int A_MN, int B_MN, int EPI>
-bool launch_bn(const Launch& L, const CUtensorMap& ma, const CUtensorMap& mb, const TcArgs& t, int bn, int m_tiles,
-               int n_tiles, int G) {
-  switch (bn) {
-    case 64: return launch<A_MN, B_MN, 64, 4, EPI>(L, ma, mb, t, m_tiles, n_tiles, G);
-    case 128: return launch<A_MN, B_MN, 128, 3, EPI>(L, ma, mb, t, m_tiles, n_tiles, G);
-    default: return launch<A_MN, B_MN, 256, 4, EPI>(L, ma, mb, t, m_tiles, n_tiles, G);
-  }
-}
-
 }  // namespace
 
-// Tile width: the widest of 256 / 128 / 64 that still gives every SM a tile; the weight-update
-// epilogue moves 10 bytes per output element, so it prefers two resident CTAs of width 128.
+// Tile width: the widest of 256 / 128 / 64 that still gives every SM a tile.  The weight-update
+// epilogue streams 10 bytes per output element and keeps its chunk ring in shared memory, so it
+// stays at 128 columns.
 int pick_bn(int M, int N, int G, int epi) {
   const long long m_tiles = ceil_div(M, BM);
   auto tiles = [&](int bn) { return m_tiles * ceil_div(N, bn) * G; };
-  if (epi == EPI_SGD) return (N > 64 && tiles(128) >= 148) ? 128 : 64;
-  if (N > 128 && tiles(256) >= 148) return 256;
-  if (N > 64 && tiles(128) >= 148) return 128;
+  const int sms = sm_count();
+  if (epi == EPI_SGD) return (N > 64 && tiles(128) >= sms) ? 128 : 64;
+  if (N > 128 && tiles(256) >= sms) return 256;
+  if (N > 64 && tiles(128) >= sms) return 128;
   return 64;
 }
 
@@ -406,45 +594,57 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
   if (!a_mn && a.a_sk != 1) return false;
   if (!b_mn && a.b_sk != 1) return false;
   const int bn = pick_bn(a.M, n_store, a.G, a.epi);
-  const int m_tiles = (int)ceil_div(a.M, BM), n_tiles = (int)ceil_div(n_store, bn);
-  if (n_tiles > 65535 || a.G > 65535) return false;
-  CUtensorMap ma, mb;
-  // K-major operand: inner = K, outer = rows (M or N).  MN-major: inner = rows, outer = K.
-  const long long ga = (a.G > 1 && a.a_sg != 0) ? a.G : 1, gb = (a.G > 1 && a.b_sg != 0) ? a.G : 1;
-  const bool ok_a = a_mn ? make_map(&ma, a.A, a.M, a.K, ga, a.a_sk, a.a_sg, BK)
-                         : make_map(&ma, a.A, a.K, a.M, ga, a.a_sm, a.a_sg, BM);
-  const bool ok_b = b_mn ? make_map(&mb, a.B, a.N, a.K, gb, a.b_sk, a.b_sg, BK)
-                         : make_map(&mb, a.B, a.K, a.N, gb, a.b_sn, a.b_sg, bn);
-  if (!ok_a || !ok_b) return false;
   TcArgs t{};
   t.M = a.M; t.N = n_store; t.K = a.K;
+  t.m_tiles = (int)ceil_div(a.M, BM);
+  t.n_tiles = (int)ceil_div(n_store, bn);
+  t.G = a.G;
   t.a_gmul = (a.G > 1 && a.a_sg != 0) ? 1 : 0;
   t.b_gmul = (a.G > 1 && a.b_sg != 0) ? 1 : 0;
-  t.epi = a.epi;
   t.bias = a.bias; t.bias_sg = a.bias_sg;
-  t.out = a.out; t.out_ld = a.out_ld; t.out_sg = a.out_sg;
-  t.outf = a.outf; t.outf_ld = a.outf_ld; t.outf_sg = a.outf_sg;
-  t.mask = a.mask; t.mask_ld = a.mask_ld; t.mask_sg = a.mask_sg;
-  t.opw = a.opw;
   t.lr = a.lr;
   t.status = st;
+  if ((long long)t.m_tiles * t.n_tiles * t.G > 0x7fffffffll) return false;
+
+  Maps m{};
+  // K-major operand: inner = K, outer = rows (M or N).  MN-major: inner = rows, outer = K.
+  const long long ga = t.a_gmul ? a.G : 1, gb = t.b_gmul ? a.G : 1;
+  const bool ok_a = a_mn ? make_map(&m.a, a.A, 2, a.M, a.K, ga, a.a_sk, a.a_sg, 64, BK, 128)
+                         : make_map(&m.a, a.A, 2, a.K, a.M, ga, a.a_sm, a.a_sg, 64, BM, 128);
+  const bool ok_b = b_mn ? make_map(&m.b, a.B, 2, a.N, a.K, gb, a.b_sk, a.b_sg, 64, BK, 128)
+                         : make_map(&m.b, a.B, 2, a.K, a.N, gb, a.b_sn, a.b_sg, 64, bn, 128);
+  if (!ok_a || !ok_b) return false;
+  m.c32 = m.a; m.c16 = m.a; m.aux16 = m.a;   // placeholders for the maps an epilogue does not use
+  // Output / epilogue-input chunks: [G][M][n_store] row-major, boxes of 128 rows x 32 columns.
   switch (a.epi) {
     case EPI_BIAS_RELU:
-      if (!a_mn && b_mn) return launch_bn<0, 1, EPI_BIAS_RELU>(L, ma, mb, t, bn, m_tiles, n_tiles, a.G);
-      break;
+      if (a_mn || !b_mn) return false;
+      if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
+      if (bn == 256) return launch<0, 1, 256, 4, 3, EPI_BIAS_RELU>(L, m, t);
+      if (bn == 128) return launch<0, 1, 128, 6, 3, EPI_BIAS_RELU>(L, m, t);
+      return launch<0, 1, 64, 8, 3, EPI_BIAS_RELU>(L, m, t);
     case EPI_BIAS_F32:
-      if (!a_mn && b_mn) return launch_bn<0, 1, EPI_BIAS_F32>(L, ma, mb, t, bn, m_tiles, n_tiles, a.G);
-      break;
+      if (a_mn || !b_mn) return false;
+      if (!make_map(&m.c32, a.outf, 4, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 128)) return false;
+      if (bn == 256) return launch<0, 1, 256, 4, 2, EPI_BIAS_F32>(L, m, t);
+      if (bn == 128) return launch<0, 1, 128, 5, 3, EPI_BIAS_F32>(L, m, t);
+      return launch<0, 1, 64, 6, 3, EPI_BIAS_F32>(L, m, t);
     case EPI_RELU_MASK:
-      if (!a_mn && !b_mn) return launch_bn<0, 0, EPI_RELU_MASK>(L, ma, mb, t, bn, m_tiles, n_tiles, a.G);
-      break;
+      if (a_mn || b_mn) return false;
+      if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
+      if (!make_map(&m.aux16, a.mask, 2, n_store, a.M, a.G, a.mask_ld, a.mask_sg, CH, BM, 64)) return false;
+      if (bn == 256) return launch<0, 0, 256, 4, 4, EPI_RELU_MASK>(L, m, t);
+      if (bn == 128) return launch<0, 0, 128, 6, 4, EPI_RELU_MASK>(L, m, t);
+      return launch<0, 0, 64, 8, 4, EPI_RELU_MASK>(L, m, t);
     case EPI_SGD:
-      if (a_mn && b_mn && a.opw) return launch_bn<1, 1, EPI_SGD>(L, ma, mb, t, bn, m_tiles, n_tiles, a.G);
-      break;
+      if (!a_mn || !b_mn || !a.opw) return false;
+      if (!make_map(&m.c32, a.outf, 4, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 128)) return false;
+      if (!make_map(&m.c16, a.opw, 2, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 64)) return false;
+      if (bn == 128) return launch<1, 1, 128, 3, 4, EPI_SGD>(L, m, t);
+      return launch<1, 1, 64, 4, 4, EPI_SGD>(L, m, t);
     default:
-      break;
+      return false;
   }
-  return false;
 }
 
 }  // namespace ist
