@@ -26,7 +26,7 @@ struct Region {
 // Placement of everything that lives in the caller's workspace blob.
 struct Plan {
   size_t total = 0;
-  Region status, keys, rank, grp, pos, row_loss, logits, ev_a, ev_b, ev_acc;
+  Region status, part, row_loss, logits, ev_a, ev_b, ev_acc;
   std::vector<Region> idx, off;             // hidden layer l at [l]  (1..t-1)
   std::vector<Region> master, bias, opw;    // layer l at [l]         (1..t)
   std::vector<Region> act, delta;           // act [0..t-1], delta [1..t]
@@ -144,10 +144,7 @@ void make_plan(ist_ctx* c) {
   int64_t maxH = 1, maxN = 0;
   for (int l = 1; l < t; ++l) maxH = std::max(maxH, c->N[l]);
   for (int l = 0; l <= t; ++l) maxN = std::max(maxN, c->N[l]);
-  p.keys = p.take(maxH * 8);
-  p.rank = p.take(maxH * 4);
-  p.grp = p.take(maxH * 4);
-  p.pos = p.take(maxH * 4);
+  p.part = p.take(partition_scratch_bytes((int)maxH, S));
   for (int l = 1; l < t; ++l) {
     p.idx[l] = p.take(c->N[l] * 4);
     p.off[l] = p.take((S + 1) * 4);
@@ -335,6 +332,18 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       if (loss_out) loss_reduce(L, row_loss, S, B, loss_out, K, k);
     }
     // ---- backward + SGD, last layer first.  delta_{l-1} is taken before W_l is updated. -----
+    auto update_biases = [&](int l_hi, int l_lo) {   // db_l = sum_b delta_l, layers l_lo..l_hi
+      Scope sc(c, IST_K_BIAS_SGD);
+      BiasSgdArgs<T> ba{};
+      int n = 0;
+      for (int l = l_hi; l >= l_lo; --l) {
+        ba.layer[n++] = BiasSgdLayer<T>{delta(l), c->ld[l], Bm * c->ld[l], c->bias(l), c->ld[l], (int)c->np[l]};
+        if (n == kMaxBiasLayers || l == l_lo) {
+          bias_sgd<T>(L, ba, n, S, B, lr);
+          n = 0;
+        }
+      }
+    };
     for (int l = t; l >= 1; --l) {
       if (l > 1) {
         GemmArgs<T> g{};
@@ -347,10 +356,6 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.out = delta(l - 1); g.out_ld = c->ld[l - 1]; g.out_sg = Bm * c->ld[l - 1];
         Scope sc(c, IST_K_DX);
         if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMM of layer %d cannot be launched", l);
-      }
-      {
-        Scope sc(c, IST_K_BIAS_SGD);
-        bias_sgd<T>(L, delta(l), c->ld[l], Bm * c->ld[l], S, B, (int)c->np[l], c->bias(l), c->ld[l], lr);
       }
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {
         Scope sc(c, IST_K_SPMM);
@@ -371,6 +376,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       Scope sc(c, IST_K_DW_SGD);
       if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "weight-gradient GEMM of layer %d cannot be launched", l);
     }
+    update_biases(t, 1);   // every delta_l is still in place; biases are not read by the backward pass
   }
   IST_CUDA(c, cudaGetLastError());
   return IST_OK;
@@ -448,9 +454,10 @@ extern "C" ist_status ist_partition(ist_ctx* c, uint64_t seed) {
   for (int l = 1; l < t; ++l) {
     Scope sc(c, IST_K_PARTITION);
     uint64_t layer_seed = splitmix64_next(&round_state);
-    partition_layer(L, layer_seed, (int)c->N[l], S, c->plan.keys.at<uint64_t>(c->ws),
-                    c->plan.rank.at<int32_t>(c->ws), c->plan.grp.at<int32_t>(c->ws),
-                    c->plan.pos.at<int32_t>(c->ws), c->idx(l), c->off(l), c->status());
+    PartitionScratch ps{};
+    partition_scratch_carve(c->plan.part.at<char>(c->ws), (int)c->N[l], S, &ps);
+    if (!partition_layer(L, layer_seed, (int)c->N[l], S, ps, c->idx(l), c->off(l), c->status()))
+      return fail(c, IST_ERR_UNSUPPORTED, "S = %d exceeds what the partition kernels support (768)", S);
   }
   for (int l = 1; l <= t; ++l) {
     Scope sc(c, IST_K_GATHER);

@@ -13,10 +13,25 @@ struct Launch {
 
 // ---- partition.cu -----------------------------------------------------------------------
 // Balanced random partition of {0..N-1} into S groups from SplitMix64 keys (see ist.h).
-// Scratch: keys [N] u64, rank [N] i32, grp [N] i32, pos [N] i32.  Outputs: idx [N], off [S+1].
-void partition_layer(const Launch& L, uint64_t layer_seed, int N, int S, uint64_t* keys,
-                     int32_t* rank, int32_t* grp, int32_t* pos, int32_t* idx, int32_t* off,
-                     DeviceStatus* st);
+// Outputs: idx [N] (group-major, ascending inside a group), off [S+1].  Scratch arrays live in
+// caller-provided memory laid out by partition_scratch_carve.
+struct PartitionScratch {
+  int log_buckets, n_buckets;
+  uint64_t* keys;     // [N]
+  uint64_t* skey;     // [N] keys grouped by bucket
+  int32_t* sidx;      // [N] their neuron indices
+  int32_t* hist;      // [n_buckets]
+  int32_t* start;     // [n_buckets + 1]
+  int32_t* cursor;    // [n_buckets]
+  int32_t* grp;       // [N]
+  int32_t* lp;        // [N] position among the block's members of the same group
+  int32_t* blkcnt;    // [ceil(N/1024)][S]
+};
+size_t partition_scratch_carve(void* base, int N, int S, PartitionScratch* out);
+size_t partition_scratch_bytes(int N, int S);
+// Returns false if S is too large for the kernels' shared-memory counters (S > 768).
+bool partition_layer(const Launch& L, uint64_t layer_seed, int N, int S, const PartitionScratch& sc,
+                     int32_t* idx, int32_t* off, DeviceStatus* st);
 
 // ---- gather_scatter.cu ------------------------------------------------------------------
 // A slice map describes how packed element (s, i, j) of a layer relates to the full matrix:
@@ -78,10 +93,17 @@ void softmax_xent(const Launch& L, const float* logits, int64_t ld, int64_t sg, 
 // loss_out[g * out_stride + k] = (1/B) sum_b row_loss[g][b]  (fixed summation order)
 void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
                  int64_t out_stride, int k);
-// bias[g][n] -= lr * sum_b delta[g][b][n]
+// bias[g][n] -= lr * sum_b delta[g][b][n] for up to kMaxBiasLayers layers in one launch.
+// delta rows are ld elements long (ld a multiple of 8, 16-byte aligned); n <= ld.
+constexpr int kMaxBiasLayers = 8;
+template <typename T> struct BiasSgdLayer {
+  const T* delta; int64_t ld, sg;
+  float* bias; int64_t bias_sg;
+  int n;
+};
+template <typename T> struct BiasSgdArgs { BiasSgdLayer<T> layer[kMaxBiasLayers]; };
 template <typename T>
-void bias_sgd(const Launch& L, const T* delta, int64_t ld, int64_t sg, int G, int B, int n,
-              float* bias, int64_t bias_sg, float lr);
+void bias_sgd(const Launch& L, const BiasSgdArgs<T>& a, int n_layers, int G, int B, float lr);
 // fp32 rows -> T rows with leading dimension ld (pad columns zero), per group row offsets.
 template <typename T>
 void stage_rows(const Launch& L, const float* X, int64_t N0, int64_t group_row_stride, int G, int B,

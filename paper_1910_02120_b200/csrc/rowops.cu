@@ -77,25 +77,49 @@ __global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int B, fl
   if (threadIdx.x == 0) loss_out[(int64_t)g * out_stride + k] = acc / (float)B;
 }
 
-// Thread per column; 8 row-lanes per column reduce through shared memory in fixed order.
-template <typename T>
-__global__ void bias_sgd_kernel(const T* __restrict__ delta, int64_t ld, int64_t sg, int B, int n,
-                                float* bias, int64_t bias_sg, float lr) {
-  __shared__ float part[8][33];
-  int g = blockIdx.y;
-  int col = blockIdx.x * 32 + threadIdx.x;
-  float acc = 0.f;
-  if (col < n) {
-    const T* d = delta + (int64_t)g * sg + col;
-    for (int b = threadIdx.y; b < B; b += 8) acc += to_float(d[(int64_t)b * ld]);
-  }
-  part[threadIdx.y][threadIdx.x] = acc;
-  __syncthreads();
-  if (threadIdx.y == 0 && col < n) {
-    float s = 0.f;
+// Bias gradient and update of every layer in one launch: blockIdx.z = layer, blockIdx.y = group,
+// blockIdx.x = block of 64 columns.  Thread (cx, ry) sums 8 adjacent columns over rows
+// ry, ry + 32, ...; the 32 partial sums of a column are added in a fixed order.
+__device__ __forceinline__ void load8(const float* p, float v[8]) {
+  float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8(const bf16* p, float v[8]) {
+  uint4 u = *reinterpret_cast<const uint4*>(p);
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-    for (int u = 0; u < 8; ++u) s += part[u][threadIdx.x];
-    bias[(int64_t)g * bias_sg + col] -= lr * s;
+  for (int i = 0; i < 4; ++i) { v[2 * i] = __low2float(h[i]); v[2 * i + 1] = __high2float(h[i]); }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int B, float lr) {
+  __shared__ float part[32][65];
+  const BiasSgdLayer<T> L = a.layer[blockIdx.z];
+  const int g = blockIdx.y;
+  const int cx = threadIdx.x & 7, ry = threadIdx.x >> 3;
+  const int c0 = blockIdx.x * 64 + cx * 8;
+  if (blockIdx.x * 64 >= L.ld) return;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (c0 < L.ld) {
+    const T* d = L.delta + (int64_t)g * L.sg + c0;
+    for (int b = ry; b < B; b += 32) {
+      float v[8];
+      load8(d + (int64_t)b * L.ld, v);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] += v[e];
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) part[ry][cx * 8 + e] = acc[e];
+  __syncthreads();
+  if (threadIdx.x < 64) {
+    const int col = blockIdx.x * 64 + threadIdx.x;
+    if (col < L.n) {
+      float s = 0.f;
+#pragma unroll
+      for (int u = 0; u < 32; ++u) s += part[u][threadIdx.x];
+      L.bias[(int64_t)g * L.bias_sg + col] -= lr * s;
+    }
   }
 }
 
@@ -190,16 +214,14 @@ void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* lo
 }
 
 template <typename T>
-void bias_sgd(const Launch& L, const T* delta, int64_t ld, int64_t sg, int G, int B, int n,
-              float* bias, int64_t bias_sg, float lr) {
-  bias_sgd_kernel<T><<<dim3((unsigned)ceil_div(n, 32), G), dim3(32, 8), 0, L.stream>>>(
-      delta, ld, sg, B, n, bias, bias_sg, lr);
+void bias_sgd(const Launch& L, const BiasSgdArgs<T>& a, int n_layers, int G, int B, float lr) {
+  int64_t max_ld = 0;
+  for (int i = 0; i < n_layers; ++i) max_ld = a.layer[i].ld > max_ld ? a.layer[i].ld : max_ld;
+  bias_sgd_kernel<T><<<dim3((unsigned)ceil_div(max_ld, 64), G, n_layers), 256, 0, L.stream>>>(a, B, lr);
   L.count();
 }
-template void bias_sgd<float>(const Launch&, const float*, int64_t, int64_t, int, int, int, float*,
-                              int64_t, float);
-template void bias_sgd<bf16>(const Launch&, const bf16*, int64_t, int64_t, int, int, int, float*,
-                             int64_t, float);
+template void bias_sgd<float>(const Launch&, const BiasSgdArgs<float>&, int, int, int, float);
+template void bias_sgd<bf16>(const Launch&, const BiasSgdArgs<bf16>&, int, int, int, float);
 
 template <typename T>
 void stage_rows(const Launch& L, const float* X, int64_t N0, int64_t group_row_stride, int G, int B,

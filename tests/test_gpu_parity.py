@@ -40,7 +40,8 @@ def _parts_equal(gp, op):
 
 @pytest.mark.parametrize("dims,S", [
     ([16, 1024, 10], 2), ([8, 1000, 777, 5], 7), ([8, 4096, 4096, 35], 4), ([4, 33, 3], 1),
-    ([4, 16, 16, 3], 16), ([8, 16384, 5], 8), ([8, 300, 301, 302, 4], 3),
+    ([4, 16, 16, 3], 16), ([8, 16384, 5], 8), ([8, 300, 301, 302, 4], 3), ([4, 5000, 3], 700),
+    ([4, 65536, 3], 16), ([4, 7, 3], 7), ([4, 1025, 1023, 3], 2),
 ])
 def test_partition_matches_oracle_bit_exact(dims, S):
     from oracle import ist_oracle as O
@@ -139,6 +140,8 @@ def test_fp32_round_tiny_config():
     ([12, 6], 1, 5, 3),                  # no hidden layer
     ([9, 40, 4], 1, 1, 2),               # S = 1, batch 1
     ([64, 256, 256, 35], 4, 64, 5),
+    ([40, 301, 10], 3, 8, 2),            # first layer wide enough for the staged column permutation, odd width
+    ([16, 2500, 6], 5, 4, 1),            # more than one staged column chunk
 ])
 def test_fp32_round_shapes(dims, S, B, K):
     _check_round(_wl("s", dims, S, B, K, "fp32", lr=0.05), FP32_RTOL, 1e-3, FP32_RTOL, True)
@@ -151,6 +154,7 @@ def test_fp32_round_shapes(dims, S, B, K):
     ([24, 100, 10], 3, 19, 3, "normal"),                   # ragged everything
     ([40, 72, 136, 200, 12], 2, 40, 2, "normal"),
     ([1024, 2048, 2048, 100], 16, 512, 2, "normal"),       # sweep shape
+    ([48, 515, 10], 4, 24, 2, "normal"),                   # staged column permutation, odd width
 ])
 def test_bf16_round_shapes(dims, S, B, K, x_dist):
     _check_round(_wl("b", dims, S, B, K, "bf16", x_dist=x_dist), BF16_W_RTOL, BF16_DW_RTOL,
