@@ -227,6 +227,26 @@ def run_reference(args, w):
 
 
 # ---------------------------------------------------------------------------------------------
+# multi-rank plumbing: replicas only, no data-path collective
+# ---------------------------------------------------------------------------------------------
+
+def max_over_ranks(ms: float, device=None) -> float:
+    """Slowest rank's elapsed time (the job is as slow as its slowest replica)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(samples_per_rank_step: int, steps: int, world: int, ms: float) -> float:
+    """Whole-job samples/s: every rank processed samples_per_rank_step * steps samples in ms."""
+    return world * samples_per_rank_step * steps / (ms * 1e-3)
+
+
+# ---------------------------------------------------------------------------------------------
 # the CUDA path
 # ---------------------------------------------------------------------------------------------
 
@@ -282,13 +302,6 @@ def run_ours(args, w):
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    def max_over_ranks(ms):
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return ms
-
     # ---- device-resident timing ---------------------------------------------------------------
     n_warm = args.warmup if args.quick else max(args.warmup, 3)
     for i in range(n_warm):
@@ -306,9 +319,9 @@ def run_ours(args, w):
     barrier()
     launches = ctx.kernel_launches() - launches0
     clocks = sampler.stop()
-    ms = max_over_ranks(e0.elapsed_time(e1))
+    ms = max_over_ranks(e0.elapsed_time(e1), dev)
     ctx.sync_status()
-    value = world * w.samples_per_round * args.steps / (ms * 1e-3)
+    value = job_value(w.samples_per_round, args.steps, world, ms)
     if args.quick:
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -336,8 +349,8 @@ def run_ours(args, w):
         e2e_round(200 + i)
     e1.record()
     barrier()
-    ms_e2e = max_over_ranks(e0.elapsed_time(e1))
-    e2e_value = world * w.samples_per_round * args.steps / (ms_e2e * 1e-3)
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1), dev)
+    e2e_value = job_value(w.samples_per_round, args.steps, world, ms_e2e)
 
     # ---- per-kernel-class device times (separate pass, events around each class) ---------------
     ctx.profile(True)
