@@ -188,6 +188,38 @@ ist_status ist_profile(ist_ctx* ctx, int enable);
 ist_status ist_profile_read(ist_ctx* ctx, int kernel_class, int64_t* launches_out_host,
                             double* ms_out_host);
 
+/*
+ * Partition of one hidden layer without a context, a workspace or any allocation.  (The paper
+ * has no counterpart; this is a service entry point of the library.)
+ *
+ * For callers that cannot obtain device memory at the time they need a partition: code running
+ * inside a host application that gave out its device-memory budget at start-up and forbids
+ * allocation afterwards, or a process that only wants the index lists (for example to decide
+ * which weight slices to fetch) and has no room for an ist_ctx workspace.  The caller passes
+ * only its own outputs; the kernels' intermediate arrays live in a device array that is part of
+ * the library image, 2 MB that every GPU loading the library holds until exit.
+ *
+ * Result: exactly the partition ist_partition(seed) draws for hidden layer `hidden_layer`
+ * (1-based) when that layer has n_neurons neurons and the network is split into S subnets:
+ * idx_out_dev [n_neurons] int32 (group-major, ascending inside a group), off_out_dev [S+1].
+ * Work is enqueued on cuda_stream (a cudaStream_t, NULL = default stream), asynchronously.
+ *
+ * Limits: n_neurons <= IST_STATIC_MAX_NEURONS and S <= IST_STATIC_MAX_SUBNETS, otherwise
+ * IST_ERR_UNSUPPORTED and nothing is enqueued.  IST_ERR_ARG for null outputs, S < 1,
+ * S > n_neurons or hidden_layer outside 1..62.  The call performs no cudaMalloc / cudaFree and
+ * calls no allocating routine.
+ *
+ * The first call on a device looks up the device address of the built-in array (a host-side
+ * set-up step): make that first call before starting any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's contents; the
+ * entry point clears what has to start at zero.  Two calls whose kernels can overlap on the
+ * GPU (different streams without an ordering between them) race on it: order them.
+ */
+#define IST_STATIC_MAX_NEURONS 65536
+#define IST_STATIC_MAX_SUBNETS 64
+ist_status ist_partition_layer_static(uint64_t seed, int hidden_layer, int64_t n_neurons, int S,
+                                      int32_t* idx_out_dev, int32_t* off_out_dev, void* cuda_stream);
+
 /* Number of kernels this context has launched so far (host counter). */
 int64_t ist_kernel_launches(const ist_ctx* ctx);
 

@@ -24,7 +24,9 @@ EXPORTS = [
     "ist_workspace_bytes", "ist_create", "ist_bind_weights", "ist_partition", "ist_get_partition",
     "ist_get_subnet_params", "ist_local_steps", "ist_reassemble", "ist_eval", "ist_sync_status",
     "ist_kernel_launches", "ist_last_error", "ist_destroy", "ist_profile", "ist_profile_read",
+    "ist_partition_layer_static",
 ]
+IST_STATIC_MAX_NEURONS, IST_STATIC_MAX_SUBNETS = 65536, 64
 
 KERNEL_CLASSES = ["partition", "gather", "stage", "fwd", "loss", "dx", "dw_sgd", "bias_sgd", "spmm",
                   "scatter", "eval"]
@@ -85,6 +87,8 @@ def _load() -> ctypes.CDLL:
     lib.ist_profile.argtypes = [vp, i32]
     lib.ist_profile_read.restype = ctypes.c_int32
     lib.ist_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double)]
+    lib.ist_partition_layer_static.restype = ctypes.c_int32
+    lib.ist_partition_layer_static.argtypes = [u64, i32, i64, i32, vp, vp, vp]
     lib.ist_destroy.restype = None
     lib.ist_destroy.argtypes = [vp]
     return lib
@@ -135,6 +139,21 @@ def make_input(X, batch: int, stride_subnet: int, stride_step: int) -> Tuple[Ist
         raise TypeError(f"unsupported input dtype {X.dtype}")
     inp.dense = X.data_ptr()
     return inp, (X,)
+
+
+def ist_partition_layer_static(seed: int, hidden_layer: int, n_neurons: int, S: int,
+                               idx_out: torch.Tensor, off_out: torch.Tensor,
+                               stream: Optional[torch.cuda.Stream] = None) -> int:
+    """Partition of one hidden layer into caller-owned int32 tensors, using the library's built-in
+    device scratch instead of a workspace (for callers that must not allocate).  Returns the
+    ist_status; work is asynchronous on `stream` (default: the current stream of idx_out's device)."""
+    assert idx_out.is_cuda and idx_out.dtype == torch.int32 and idx_out.numel() >= n_neurons
+    assert off_out.is_cuda and off_out.dtype == torch.int32 and off_out.numel() >= S + 1
+    with torch.cuda.device(idx_out.device):
+        s = stream if stream is not None else torch.cuda.current_stream(idx_out.device)
+        return int(lib.ist_partition_layer_static(ctypes.c_uint64(seed & (2 ** 64 - 1)), hidden_layer, n_neurons, S,
+                                                  idx_out.data_ptr(), off_out.data_ptr(),
+                                                  ctypes.c_void_p(s.cuda_stream)))
 
 
 class Ist:
