@@ -12,7 +12,7 @@ from typing import List, Optional, Sequence, Tuple
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libist.so")
+LIB_PATH = os.environ.get("IST_LIB_PATH") or os.path.join(_HERE, "libist.so")
 
 IST_OK = 0
 IST_ERR_ARG, IST_ERR_STATE, IST_ERR_WORKSPACE, IST_ERR_CUDA = -1, -2, -3, -4

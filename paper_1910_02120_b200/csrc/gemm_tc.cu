@@ -20,6 +20,12 @@
 // 2*B flops): its fp32 master chunks are prefetched through a ring several chunks deep while
 // earlier chunks are updated in place in shared memory and stored back.
 //
+// PAIR = 2 runs two CTAs of a cluster as one unit (tcgen05 cta_group::2): the pair computes a
+// 256 x BN tile, each CTA loads its own 128 rows of A and its half (BN/2 rows) of B and keeps its
+// own 128 x BN accumulator, and the leader CTA (cluster rank 0) issues one MMA that reads both
+// CTAs' shared memory.  Every B byte then enters shared memory once per 256 output rows instead
+// of once per 128, which is what the L2-to-SM path needs to keep the tensor pipe fed.
+//
 // Either operand may be contiguous along k ("K-major") or along m/n ("MN-major"); the shared
 // memory tile is 128-byte swizzled in both cases and the UMMA descriptors say which.  Rows and
 // columns beyond the tensor extents are zero-filled by TMA loads and dropped by TMA stores.
@@ -94,6 +100,33 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+// Same copy issued by a CTA of a pair; the mbarrier may live in the peer CTA (shared::cluster
+// address), which is how both CTAs' loads complete on the leader's "full" barrier.
+__device__ __forceinline__ void tma_load_3d_pair(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
+                                                 int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* src, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
                ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2)
@@ -126,6 +159,23 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
+}
+// Pair forms: one commit arrives on the barrier at the same offset in both CTAs; one MMA
+// reads both CTAs' operand tiles and writes both accumulators.
+__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(smem_u32(bar)), "h"((uint16_t)3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
 }
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                        uint32_t accumulate) {
@@ -163,9 +213,9 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 
 // Instruction descriptor: D = f32 (bits 4..5 = 1), A and B = bf16 (bits 7..9, 10..12 = 1),
 // operand majors (bit 15 / 16: 1 = MN-major), N >> 3 at bits 17..22, M >> 4 at bits 24..28.
-__host__ __device__ constexpr uint32_t make_idesc(int a_mn, int b_mn, int n) {
+__host__ __device__ constexpr uint32_t make_idesc(int a_mn, int b_mn, int n, int m) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 struct TcArgs {
@@ -212,7 +262,7 @@ __device__ __forceinline__ uint4* b16_unit(uint8_t* area, int r, int u) {
   return reinterpret_cast<uint4*>(area + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
 }
 
-template <int A_MN, int B_MN, int BN, int STAGES, int N32, int N16, int EPI>
+template <int A_MN, int B_MN, int BN, int STAGES, int N32, int N16, int EPI, int PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC32,   // fp32 chunks: logits out, master in/out
@@ -221,7 +271,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                TcArgs a) {
   using ET = EpiTraits<EPI>;
   static_assert(ET::k32 == (N32 > 0) && ET::k16 == (N16 > 0), "ring sizes do not match the epilogue");
-  constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int BNL = BN / PAIR;   // rows of the B tile this CTA loads
+  constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BNL * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
   constexpr uint32_t F32_BYTES = BM * CH * 4, B16_BYTES = BM * CH * 2;
   constexpr int NAUX = EPI == EPI_SGD ? N32 : (EPI == EPI_RELU_MASK ? N16 : 1);
   constexpr uint32_t AUX_BYTES = EPI == EPI_SGD ? F32_BYTES : B16_BYTES;
@@ -242,7 +293,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (a.K + BK - 1) / BK;
-  const int total_tiles = a.m_tiles * a.n_tiles * a.G;
+  const int total_tiles = a.m_tiles * a.n_tiles * a.G;   // tiles of (128 * PAIR) x BN
+  const int rank = PAIR == 2 ? (int)cluster_ctarank() : 0;
+  const int unit = blockIdx.x / PAIR, n_units = gridDim.x / PAIR;   // a unit = a CTA or a pair
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -251,7 +304,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&acc_full[b], 1);
-      mbar_init(&acc_empty[b], kEpiThreads / 32);   // one arrival per epilogue warp
+      mbar_init(&acc_empty[b], PAIR * kEpiThreads / 32);   // one arrival per epilogue warp of the unit
     }
     for (int s = 0; s < NAUX; ++s) {
       mbar_init(&slot_full[s], 1);
@@ -262,13 +315,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     fence_async_smem();
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR == 2) cluster_sync_all();   // the peer's barriers are initialised before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot;
   volatile int* abortp = &abort_flag;
@@ -278,9 +339,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) {
       int it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile % a.m_tiles) * BM;
-        const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
+      for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
+        const int m0 = (tile % a.m_tiles) * (BM * PAIR) + rank * BM;     // this CTA's rows of A
+        const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN + rank * BNL;   // this CTA's rows of B
         const int g = tile / (a.m_tiles * a.n_tiles);
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % STAGES;
@@ -288,25 +349,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (!ok) break;
           uint8_t* sa = smem + s * STAGE_BYTES;
           uint8_t* sb = sa + A_BYTES;
-          mbar_expect_tx(&full_bar[s], STAGE_BYTES);
-          if (A_MN) {
+          if (PAIR == 2) {
+            // both CTAs' copies complete on the leader's barrier, which expects the bytes of both
+            const uint32_t bar = map_to_cta(&full_bar[s], 0);
+            if (rank == 0) mbar_expect_tx(&full_bar[s], 2 * STAGE_BYTES);
+            if (A_MN) {
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j)
-              tma_load_3d(sa + j * (BK * 128), &tmA, &full_bar[s], m0 + 64 * j, kb * BK, g * a.a_gmul);
-          } else {
-            tma_load_3d(sa, &tmA, &full_bar[s], kb * BK, m0, g * a.a_gmul);
-          }
-          if (B_MN) {
+              for (int j = 0; j < BM / 64; ++j)
+                tma_load_3d_pair(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, kb * BK, g * a.a_gmul);
+            } else {
+              tma_load_3d_pair(sa, &tmA, bar, kb * BK, m0, g * a.a_gmul);
+            }
+            if (B_MN) {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j)
-              tma_load_3d(sb + j * (BK * 128), &tmB, &full_bar[s], n0 + 64 * j, kb * BK, g * a.b_gmul);
+              for (int j = 0; j < BNL / 64; ++j)
+                tma_load_3d_pair(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, kb * BK, g * a.b_gmul);
+            } else {
+              tma_load_3d_pair(sb, &tmB, bar, kb * BK, n0, g * a.b_gmul);
+            }
           } else {
-            tma_load_3d(sb, &tmB, &full_bar[s], kb * BK, n0, g * a.b_gmul);
+            mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+            if (A_MN) {
+#pragma unroll
+              for (int j = 0; j < BM / 64; ++j)
+                tma_load_3d(sa + j * (BK * 128), &tmA, &full_bar[s], m0 + 64 * j, kb * BK, g * a.a_gmul);
+            } else {
+              tma_load_3d(sa, &tmA, &full_bar[s], kb * BK, m0, g * a.a_gmul);
+            }
+            if (B_MN) {
+#pragma unroll
+              for (int j = 0; j < BNL / 64; ++j)
+                tma_load_3d(sb + j * (BK * 128), &tmB, &full_bar[s], n0 + 64 * j, kb * BK, g * a.b_gmul);
+            } else {
+              tma_load_3d(sb, &tmB, &full_bar[s], kb * BK, n0, g * a.b_gmul);
+            }
           }
         }
       }
-      if (!ok) {
-        // let copies already in flight land before the CTA's shared memory goes away
+      if (!ok && rank == 0) {
+        // let copies already in flight land before the CTA's shared memory goes away (a peer CTA
+        // is held by the closing cluster barrier until the leader has got here)
         for (int j = max(0, it - STAGES); j < it; ++j) {
           long long t0 = clock64();
           while (!mbar_try_wait(&full_bar[j % STAGES], (j / STAGES) & 1) && clock64() - t0 < kWaitLimitCycles) {}
@@ -315,11 +397,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issue
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BN);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BN, BM * PAIR);
       int it = 0, j = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++j) {
+      for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
         const int b = j & 1;
         ok = mbar_wait(&acc_empty[b], ((j >> 1) & 1) ^ 1, abortp, a.status, 2);
         if (!ok) break;
@@ -337,11 +419,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // MN-major: 16 k-rows = 2048 B; 64-element MN chunks (one TMA box each) 8192 B apart.
             const uint64_t ad = A_MN ? make_desc(sa + k * 2048, BK * 128, 1024) : make_desc(sa + k * 32, 16, 1024);
             const uint64_t bd = B_MN ? make_desc(sb + k * 2048, BK * 128, 1024) : make_desc(sb + k * 32, 16, 1024);
-            tc_mma(d_tmem, ad, bd, idesc, (kb | k) != 0);
+            if (PAIR == 2) tc_mma_pair(d_tmem, ad, bd, idesc, (kb | k) != 0);
+            else tc_mma(d_tmem, ad, bd, idesc, (kb | k) != 0);
           }
-          tc_commit(&empty_bar[s]);   // frees the slot once these MMAs have read it
+          // frees the slot (in both CTAs of a pair) once these MMAs have read it
+          if (PAIR == 2) tc_commit_pair(&empty_bar[s]); else tc_commit(&empty_bar[s]);
         }
-        if (ok) tc_commit(&acc_full[b]);
+        if (ok) {
+          if (PAIR == 2) tc_commit_pair(&acc_full[b]); else tc_commit(&acc_full[b]);
+        }
       }
     }
   } else if (warp < kAuxWarp) {
@@ -352,8 +438,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool leader = threadIdx.x == 64;            // issues the TMA stores
     int cq = 0, j = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++j) {
-      const int m0 = (tile % a.m_tiles) * BM;
+    for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
+      const int m0 = (tile % a.m_tiles) * (BM * PAIR) + rank * BM;
       const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
       const int g = tile / (a.m_tiles * a.n_tiles);
       const int b = j & 1;
@@ -442,7 +528,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) break;
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&acc_empty[b]);
+      if (lane == 0) {   // the accumulator is free again: tell the CTA that issues the MMAs
+        if (PAIR == 2) mbar_arrive_cluster(map_to_cta(&acc_empty[b], 0)); else mbar_arrive(&acc_empty[b]);
+      }
     }
     if (leader) tma_wait_all();      // all stores complete before the CTA exits
   } else {
@@ -450,8 +538,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (ET::kAux && lane == 0) {
       int cq = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile % a.m_tiles) * BM;
+      for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
+        const int m0 = (tile % a.m_tiles) * (BM * PAIR) + rank * BM;
         const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
         const int g = tile / (a.m_tiles * a.n_tiles);
         for (int c = 0; c < NCH; ++c, ++cq) {
@@ -475,10 +563,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR == 2) cluster_sync_all();   // neither CTA leaves while the other may still touch its memory
   if (warp == 1) {
     __syncwarp();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
-                 : "memory");
+    if (PAIR == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
+                   : "memory");
   }
 }
 
@@ -557,36 +650,67 @@ struct Maps {
   CUtensorMap a, b, c32, c16, aux16;
 };
 
-template <int A_MN, int B_MN, int BN, int STAGES, int N32, int N16, int EPI>
+template <int A_MN, int B_MN, int BN, int STAGES, int N32, int N16, int EPI, int PAIR>
 bool launch(const Launch& L, const Maps& m, const TcArgs& t) {
-  constexpr int smem = STAGES * (BM * BK * 2 + BN * BK * 2) + N32 * BM * CH * 4 + N16 * BM * CH * 2 + 1024;
+  constexpr int smem = STAGES * (BM * BK * 2 + (BN / PAIR) * BK * 2) + N32 * BM * CH * 4 + N16 * BM * CH * 2 + 1024;
   static_assert(smem <= 227 * 1024 - 512, "shared memory budget exceeded");
-  auto kern = gemm_tc_kernel<A_MN, B_MN, BN, STAGES, N32, N16, EPI>;
-  static bool configured = false;
-  if (!configured) {
+  auto kern = gemm_tc_kernel<A_MN, B_MN, BN, STAGES, N32, N16, EPI, PAIR>;
+  static int max_units = 0;   // CTAs (PAIR = 1) or clusters (PAIR = 2) that can be resident at once
+  if (max_units == 0) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-    configured = true;
+    if (PAIR == 2) {
+      cudaLaunchConfig_t probe{};
+      probe.gridDim = dim3(2 * (sm_count() / 2));
+      probe.blockDim = dim3(kThreads);
+      probe.dynamicSmemBytes = smem;
+      cudaLaunchAttribute attr{};
+      attr.id = cudaLaunchAttributeClusterDimension;
+      attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+      probe.attrs = &attr;
+      probe.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &probe) != cudaSuccess || n <= 0) return false;
+      max_units = n < sm_count() / 2 ? n : sm_count() / 2;
+    } else {
+      max_units = sm_count();
+    }
   }
   const int total = t.m_tiles * t.n_tiles * t.G;
-  const int grid = total < sm_count() ? total : sm_count();
-  kern<<<grid, kThreads, smem, L.stream>>>(m.a, m.b, m.c32, m.c16, m.aux16, t);
+  const int units = total < max_units ? total : max_units;
+  if (PAIR == 2) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * units);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = L.stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, m.a, m.b, m.c32, m.c16, m.aux16, t) != cudaSuccess) return false;
+  } else {
+    kern<<<units, kThreads, smem, L.stream>>>(m.a, m.b, m.c32, m.c16, m.aux16, t);
+  }
   L.count();
   return true;
 }
 
 }  // namespace
 
-// Tile width: the widest of 256 / 128 / 64 that still gives every SM a tile.  The weight-update
-// epilogue streams 10 bytes per output element and keeps its chunk ring in shared memory, so it
-// stays at 128 columns.
-int pick_bn(int M, int N, int G, int epi) {
-  const long long m_tiles = ceil_div(M, BM);
-  auto tiles = [&](int bn) { return m_tiles * ceil_div(N, bn) * G; };
+// Tile shape.  Pairs of CTAs (256 x 256 tiles) are used when the problem has enough of them to
+// give every SM pair work; otherwise single CTAs with the widest of 256 / 128 / 64 columns that
+// still gives every SM a tile.  The weight-update epilogue keeps a chunk ring in shared memory
+// and stays at 128 columns when it runs on single CTAs.
+struct TileChoice { int bn, pair; };
+TileChoice pick_tile(int M, int N, int G, int epi) {
   const int sms = sm_count();
-  if (epi == EPI_SGD) return (N > 64 && tiles(128) >= sms) ? 128 : 64;
-  if (N > 128 && tiles(256) >= sms) return 256;
-  if (N > 64 && tiles(128) >= sms) return 128;
-  return 64;
+  auto tiles = [&](int bm, int bn) { return ceil_div(M, bm) * ceil_div(N, bn) * G; };
+  if (M > BM && N > 128 && 4 * tiles(2 * BM, 256) >= 3 * (sms / 2)) return {256, 2};
+  if (epi == EPI_SGD) return {(N > 64 && tiles(BM, 128) >= sms) ? 128 : 64, 1};
+  if (N > 128 && tiles(BM, 256) >= sms) return {256, 1};
+  if (N > 64 && tiles(BM, 128) >= sms) return {128, 1};
+  return {64, 1};
 }
 
 bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
@@ -594,10 +718,11 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
   const bool a_mn = a.a_sm == 1 && a.a_sk != 1, b_mn = a.b_sn == 1 && a.b_sk != 1;
   if (!a_mn && a.a_sk != 1) return false;
   if (!b_mn && a.b_sk != 1) return false;
-  const int bn = pick_bn(a.M, n_store, a.G, a.epi);
+  const TileChoice tc = pick_tile(a.M, n_store, a.G, a.epi);
+  const int bn = tc.bn, pair = tc.pair;
   TcArgs t{};
   t.M = a.M; t.N = n_store; t.K = a.K;
-  t.m_tiles = (int)ceil_div(a.M, BM);
+  t.m_tiles = (int)ceil_div(a.M, BM * pair);
   t.n_tiles = (int)ceil_div(n_store, bn);
   t.G = a.G;
   t.a_gmul = (a.G > 1 && a.a_sg != 0) ? 1 : 0;
@@ -613,7 +738,7 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
   const bool ok_a = a_mn ? make_map(&m.a, a.A, 2, a.M, a.K, ga, a.a_sk, a.a_sg, 64, BK, 128)
                          : make_map(&m.a, a.A, 2, a.K, a.M, ga, a.a_sm, a.a_sg, 64, BM, 128);
   const bool ok_b = b_mn ? make_map(&m.b, a.B, 2, a.N, a.K, gb, a.b_sk, a.b_sg, 64, BK, 128)
-                         : make_map(&m.b, a.B, 2, a.K, a.N, gb, a.b_sn, a.b_sg, 64, bn, 128);
+                         : make_map(&m.b, a.B, 2, a.K, a.N, gb, a.b_sn, a.b_sg, 64, bn / pair, 128);
   if (!ok_a || !ok_b) return false;
   m.c32 = m.a; m.c16 = m.a; m.aux16 = m.a;   // placeholders for the maps an epilogue does not use
   // Output / epilogue-input chunks: [G][M][n_store] row-major, boxes of 128 rows x 32 columns.
@@ -621,28 +746,32 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
     case EPI_BIAS_RELU:
       if (a_mn || !b_mn) return false;
       if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
-      if (bn == 256) return launch<0, 1, 256, 4, 0, 3, EPI_BIAS_RELU>(L, m, t);
-      if (bn == 128) return launch<0, 1, 128, 6, 0, 3, EPI_BIAS_RELU>(L, m, t);
-      return launch<0, 1, 64, 8, 0, 3, EPI_BIAS_RELU>(L, m, t);
+      if (pair == 2) return launch<0, 1, 256, 6, 0, 3, EPI_BIAS_RELU, 2>(L, m, t);
+      if (bn == 256) return launch<0, 1, 256, 4, 0, 3, EPI_BIAS_RELU, 1>(L, m, t);
+      if (bn == 128) return launch<0, 1, 128, 6, 0, 3, EPI_BIAS_RELU, 1>(L, m, t);
+      return launch<0, 1, 64, 8, 0, 3, EPI_BIAS_RELU, 1>(L, m, t);
     case EPI_BIAS_F32:
       if (a_mn || !b_mn) return false;
       if (!make_map(&m.c32, a.outf, 4, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 128)) return false;
-      if (bn == 256) return launch<0, 1, 256, 4, 2, 0, EPI_BIAS_F32>(L, m, t);
-      if (bn == 128) return launch<0, 1, 128, 5, 3, 0, EPI_BIAS_F32>(L, m, t);
-      return launch<0, 1, 64, 6, 3, 0, EPI_BIAS_F32>(L, m, t);
+      if (pair == 2) return launch<0, 1, 256, 6, 2, 0, EPI_BIAS_F32, 2>(L, m, t);
+      if (bn == 256) return launch<0, 1, 256, 4, 2, 0, EPI_BIAS_F32, 1>(L, m, t);
+      if (bn == 128) return launch<0, 1, 128, 5, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
+      return launch<0, 1, 64, 6, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
     case EPI_RELU_MASK:
       if (a_mn || b_mn) return false;
       if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
       if (!make_map(&m.aux16, a.mask, 2, n_store, a.M, a.G, a.mask_ld, a.mask_sg, CH, BM, 64)) return false;
-      if (bn == 256) return launch<0, 0, 256, 4, 0, 4, EPI_RELU_MASK>(L, m, t);
-      if (bn == 128) return launch<0, 0, 128, 6, 0, 4, EPI_RELU_MASK>(L, m, t);
-      return launch<0, 0, 64, 8, 0, 4, EPI_RELU_MASK>(L, m, t);
+      if (pair == 2) return launch<0, 0, 256, 6, 0, 4, EPI_RELU_MASK, 2>(L, m, t);
+      if (bn == 256) return launch<0, 0, 256, 4, 0, 4, EPI_RELU_MASK, 1>(L, m, t);
+      if (bn == 128) return launch<0, 0, 128, 6, 0, 4, EPI_RELU_MASK, 1>(L, m, t);
+      return launch<0, 0, 64, 8, 0, 4, EPI_RELU_MASK, 1>(L, m, t);
     case EPI_SGD:
       if (!a_mn || !b_mn || !a.opw) return false;
       if (!make_map(&m.c32, a.outf, 4, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 128)) return false;
       if (!make_map(&m.c16, a.opw, 2, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 64)) return false;
-      if (bn == 128) return launch<1, 1, 128, 4, 4, 3, EPI_SGD>(L, m, t);
-      return launch<1, 1, 64, 5, 4, 3, EPI_SGD>(L, m, t);
+      if (pair == 2) return launch<1, 1, 256, 4, 4, 3, EPI_SGD, 2>(L, m, t);
+      if (bn == 128) return launch<1, 1, 128, 4, 4, 3, EPI_SGD, 1>(L, m, t);
+      return launch<1, 1, 64, 5, 4, 3, EPI_SGD, 1>(L, m, t);
     default:
       return false;
   }

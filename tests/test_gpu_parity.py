@@ -155,6 +155,9 @@ def test_fp32_round_shapes(dims, S, B, K):
     ([40, 72, 136, 200, 12], 2, 40, 2, "normal"),
     ([1024, 2048, 2048, 100], 16, 512, 2, "normal"),       # sweep shape
     ([48, 515, 10], 4, 24, 2, "normal"),                   # staged column permutation, odd width
+    ([256, 8192, 1000], 8, 512, 2, "normal"),              # large enough for CTA-pair tiles in every GEMM
+    ([256, 8192, 8192, 10], 8, 512, 2, "normal"),
+    ([264, 6144, 2056, 24], 3, 384, 2, "normal"),          # CTA pairs with ragged edges (M = 384 = 1.5 pair tiles)
 ])
 def test_bf16_round_shapes(dims, S, B, K, x_dist):
     _check_round(_wl("b", dims, S, B, K, "bf16", x_dist=x_dist), BF16_W_RTOL, BF16_DW_RTOL,
