@@ -333,6 +333,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot;
   volatile int* abortp = &abort_flag;
+  // Programmatic dependent launch: everything above touched only this CTA's own shared and tensor
+  // memory, so it may run while the previous kernel in the stream is still draining.  From here on
+  // global memory written by that kernel is read (and buffers it reads are overwritten), so wait
+  // until it has completed and its writes are visible; then let the next kernel's CTAs be
+  // scheduled as this grid's CTAs retire.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     // ---------------------------------------------------------------- operand loads
@@ -677,21 +684,25 @@ bool launch(const Launch& L, const Maps& m, const TcArgs& t) {
   }
   const int total = t.m_tiles * t.n_tiles * t.G;
   const int units = total < max_units ? total : max_units;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(PAIR * units);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = L.stream;
+  cudaLaunchAttribute attrs[2];
+  int n_attrs = 0;
+  // the kernel's prologue may overlap the tail of the kernel before it (see griddepcontrol.wait)
+  attrs[n_attrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[n_attrs].val.programmaticStreamSerializationAllowed = 1;
+  ++n_attrs;
   if (PAIR == 2) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(2 * units);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = L.stream;
-    cudaLaunchAttribute attr{};
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, m.a, m.b, m.c32, m.c16, m.aux16, t) != cudaSuccess) return false;
-  } else {
-    kern<<<units, kThreads, smem, L.stream>>>(m.a, m.b, m.c32, m.c16, m.aux16, t);
+    attrs[n_attrs].id = cudaLaunchAttributeClusterDimension;
+    attrs[n_attrs].val.clusterDim.x = 2; attrs[n_attrs].val.clusterDim.y = 1; attrs[n_attrs].val.clusterDim.z = 1;
+    ++n_attrs;
   }
+  cfg.attrs = attrs;
+  cfg.numAttrs = n_attrs;
+  if (cudaLaunchKernelEx(&cfg, kern, m.a, m.b, m.c32, m.c16, m.aux16, t) != cudaSuccess) return false;
   L.count();
   return true;
 }
