@@ -33,6 +33,29 @@ __device__ __forceinline__ void report(DeviceStatus* st, int code, int site, lon
   }
 }
 
+// Programmatic dependent launch.  A kernel launched with launch_pdl may be scheduled while the
+// kernel before it in the stream is still running; it must call pdl_wait() before it touches
+// global memory (that waits until the earlier kernel has completed and its writes are visible).
+// pdl_trigger() lets the kernel after this one be scheduled as this grid's CTAs retire.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __host__ __device__ __forceinline__ constexpr int64_t ceil_div(int64_t a, int64_t b) {
   return (a + b - 1) / b;
 }

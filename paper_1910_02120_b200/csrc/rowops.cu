@@ -44,6 +44,8 @@ __global__ void softmax_xent_kernel(const float* __restrict__ logits, int64_t ld
                                     T* __restrict__ delta, int64_t ld_d, int64_t sg_d,
                                     float* __restrict__ row_loss, DeviceStatus* st) {
   __shared__ float sh[32];
+  pdl_wait();
+  pdl_trigger();
   int g = blockIdx.y, b = blockIdx.x;
   const float* z = logits + (int64_t)g * sg + (int64_t)b * ld;
   T* d = delta + (int64_t)g * sg_d + (int64_t)b * ld_d;
@@ -70,6 +72,8 @@ __global__ void softmax_xent_kernel(const float* __restrict__ logits, int64_t ld
 __global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int B, float* loss_out,
                                    int64_t out_stride, int k) {
   __shared__ float sh[32];
+  pdl_wait();
+  pdl_trigger();
   int g = blockIdx.x;
   float acc = 0.f;
   for (int b = threadIdx.x; b < B; b += blockDim.x) acc += row_loss[(int64_t)g * B + b];
@@ -94,6 +98,8 @@ __device__ __forceinline__ void load8(const bf16* p, float v[8]) {
 template <typename T>
 __global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int B, float lr) {
   __shared__ float part[32][65];
+  pdl_wait();
+  pdl_trigger();
   const BiasSgdLayer<T> L = a.layer[blockIdx.z];
   const int g = blockIdx.y;
   const int cx = threadIdx.x & 7, ry = threadIdx.x >> 3;
@@ -126,6 +132,8 @@ __global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int B, 
 template <typename T>
 __global__ void stage_rows_kernel(const float* __restrict__ X, int64_t N0, int64_t group_row_stride,
                                   int B, T* __restrict__ out, int64_t ld, int64_t sg) {
+  pdl_wait();
+  pdl_trigger();
   int g = blockIdx.z, b = blockIdx.y;
   int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= ld) return;
@@ -196,8 +204,8 @@ template <typename T>
 void softmax_xent(const Launch& L, const float* logits, int64_t ld, int64_t sg, int G, int B, int Nt,
                   const int32_t* y, int64_t y_sg, T* delta, int64_t ld_d, int64_t sg_d,
                   float* row_loss, DeviceStatus* st) {
-  softmax_xent_kernel<T><<<dim3(B, G), row_threads(Nt), 0, L.stream>>>(
-      logits, ld, sg, B, Nt, y, y_sg, delta, ld_d, sg_d, row_loss, st);
+  launch_pdl(softmax_xent_kernel<T>, dim3(B, G), dim3(row_threads(Nt)), 0, L.stream, logits, ld, sg, B, Nt, y, y_sg,
+             delta, ld_d, sg_d, row_loss, st);
   L.count();
 }
 template void softmax_xent<float>(const Launch&, const float*, int64_t, int64_t, int, int, int,
@@ -209,7 +217,7 @@ template void softmax_xent<bf16>(const Launch&, const float*, int64_t, int64_t, 
 
 void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
                  int64_t out_stride, int k) {
-  loss_reduce_kernel<<<G, 256, 0, L.stream>>>(row_loss, B, loss_out, out_stride, k);
+  launch_pdl(loss_reduce_kernel, dim3(G), dim3(256), 0, L.stream, row_loss, B, loss_out, out_stride, k);
   L.count();
 }
 
@@ -217,7 +225,7 @@ template <typename T>
 void bias_sgd(const Launch& L, const BiasSgdArgs<T>& a, int n_layers, int G, int B, float lr) {
   int64_t max_ld = 0;
   for (int i = 0; i < n_layers; ++i) max_ld = a.layer[i].ld > max_ld ? a.layer[i].ld : max_ld;
-  bias_sgd_kernel<T><<<dim3((unsigned)ceil_div(max_ld, 64), G, n_layers), 256, 0, L.stream>>>(a, B, lr);
+  launch_pdl(bias_sgd_kernel<T>, dim3((unsigned)ceil_div(max_ld, 64), G, n_layers), dim3(256), 0, L.stream, a, B, lr);
   L.count();
 }
 template void bias_sgd<float>(const Launch&, const BiasSgdArgs<float>&, int, int, int, float);
@@ -226,8 +234,8 @@ template void bias_sgd<bf16>(const Launch&, const BiasSgdArgs<bf16>&, int, int, 
 template <typename T>
 void stage_rows(const Launch& L, const float* X, int64_t N0, int64_t group_row_stride, int G, int B,
                 T* out, int64_t ld, int64_t sg) {
-  stage_rows_kernel<T><<<dim3((unsigned)ceil_div(ld, 256), B, G), 256, 0, L.stream>>>(
-      X, N0, group_row_stride, B, out, ld, sg);
+  launch_pdl(stage_rows_kernel<T>, dim3((unsigned)ceil_div(ld, 256), B, G), dim3(256), 0, L.stream, X, N0,
+             group_row_stride, B, out, ld, sg);
   L.count();
 }
 template void stage_rows<float>(const Launch&, const float*, int64_t, int64_t, int, int, float*,
