@@ -332,21 +332,35 @@ def run_ours(args, w):
         return
 
     # ---- end to end: host buffers in, loss out, copies inside the timed region ------------------
-    stage_in = [torch.empty_like(t, device=dev) for t in host_in]
-    stage_y = torch.empty_like(y_host, device=dev)
+    # Every round's X and y come from pinned host memory and its loss array goes back to the host.
+    # Two device staging sets: the copy of round i+1 (copy stream) overlaps the compute of round i.
+    stages = [([torch.empty_like(t, device=dev) for t in host_in], torch.empty_like(y_host, device=dev))
+              for _ in range(2)]
+    copy_stream = torch.cuda.Stream(device=dev)
+    main_stream = torch.cuda.current_stream(dev)
+    copied = [torch.cuda.Event() for _ in range(2)]
+    consumed = [torch.cuda.Event() for _ in range(2)]
 
-    def e2e_round(r):
-        for dst, src in zip(stage_in, host_in):
-            dst.copy_(src, non_blocking=True)
-        stage_y.copy_(y_host, non_blocking=True)
-        one_round(r, X_of(stage_in), stage_y)
-        loss_host.copy_(loss_dev, non_blocking=True)
+    def e2e_rounds(n, seed0):
+        for i in range(n):
+            xs, ys = stages[i % 2]
+            with torch.cuda.stream(copy_stream):
+                if i >= 2:
+                    copy_stream.wait_event(consumed[i % 2])     # round i-2 has finished with this set
+                for dst, src in zip(xs, host_in):
+                    dst.copy_(src, non_blocking=True)
+                ys.copy_(y_host, non_blocking=True)
+                copied[i % 2].record(copy_stream)
+            main_stream.wait_event(copied[i % 2])
+            one_round(seed0 + i, X_of(xs), ys)
+            consumed[i % 2].record(main_stream)
+            loss_host.copy_(loss_dev, non_blocking=True)
 
-    e2e_round(0)
+    e2e_rounds(2, 0)
     barrier()
     e0.record()
-    for i in range(args.steps):
-        e2e_round(200 + i)
+    copy_stream.wait_event(e0)          # the first copy starts inside the timed region
+    e2e_rounds(args.steps, 200)
     e1.record()
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1), dev)
