@@ -221,6 +221,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int a_mn, int b_mn, int n, int
 struct TcArgs {
   int M, N, K;            // M, N: bounds of the output rows / columns the epilogue touches
   int m_tiles, n_tiles, G;
+  int k_splits, kb_per_split;   // the k range may be cut into slices that run as separate tiles
   int a_gmul, b_gmul;     // 1 if the operand has one slab per group, 0 if all groups share it
   const float* bias; long long bias_sg;
   float lr;
@@ -293,7 +294,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (a.K + BK - 1) / BK;
-  const int total_tiles = a.m_tiles * a.n_tiles * a.G;   // tiles of (128 * PAIR) x BN
+  const int total_tiles = a.m_tiles * a.n_tiles * a.G * a.k_splits;   // tiles of (128 * PAIR) x BN x k slice
   const int rank = PAIR == 2 ? (int)cluster_ctarank() : 0;
   const int unit = blockIdx.x / PAIR, n_units = gridDim.x / PAIR;   // a unit = a CTA or a pair
 
@@ -349,8 +350,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
         const int m0 = (tile % a.m_tiles) * (BM * PAIR) + rank * BM;     // this CTA's rows of A
         const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN + rank * BNL;   // this CTA's rows of B
-        const int g = tile / (a.m_tiles * a.n_tiles);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const int rest = tile / (a.m_tiles * a.n_tiles);
+        const int g = rest / a.k_splits;
+        const int kb0 = (rest % a.k_splits) * a.kb_per_split, kb1 = min(num_kb, kb0 + a.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           ok = mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abortp, a.status, 1);
           if (!ok) break;
@@ -414,7 +417,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const int kb0 = ((tile / (a.m_tiles * a.n_tiles)) % a.k_splits) * a.kb_per_split;
+        const int kb1 = min(num_kb, kb0 + a.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           ok = mbar_wait(&full_bar[s], (it / STAGES) & 1, abortp, a.status, 3);
           if (!ok) break;
@@ -426,8 +431,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // MN-major: 16 k-rows = 2048 B; 64-element MN chunks (one TMA box each) 8192 B apart.
             const uint64_t ad = A_MN ? make_desc(sa + k * 2048, BK * 128, 1024) : make_desc(sa + k * 32, 16, 1024);
             const uint64_t bd = B_MN ? make_desc(sb + k * 2048, BK * 128, 1024) : make_desc(sb + k * 32, 16, 1024);
-            if (PAIR == 2) tc_mma_pair(d_tmem, ad, bd, idesc, (kb | k) != 0);
-            else tc_mma(d_tmem, ad, bd, idesc, (kb | k) != 0);
+            if (PAIR == 2) tc_mma_pair(d_tmem, ad, bd, idesc, ((kb - kb0) | k) != 0);
+            else tc_mma(d_tmem, ad, bd, idesc, ((kb - kb0) | k) != 0);
           }
           // frees the slot (in both CTAs of a pair) once these MMAs have read it
           if (PAIR == 2) tc_commit_pair(&empty_bar[s]); else tc_commit(&empty_bar[s]);
@@ -495,14 +500,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             *pm = pack8(o);
           }
         } else {
-          const float* bias = a.bias + (long long)g * a.bias_sg;
+          // bias of the tile's group; a k slice of a split product carries none
+          const float* bias = a.bias ? a.bias + (long long)(g / a.k_splits) * a.bias_sg : nullptr;
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
             float o[8];
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
               const int n = nc + 16 * h + 8 * u + 4 * hh;
-              float4 bv = n < a.N ? __ldg(reinterpret_cast<const float4*>(bias + n)) : make_float4(0.f, 0.f, 0.f, 0.f);
+              float4 bv = (bias && n < a.N) ? __ldg(reinterpret_cast<const float4*>(bias + n))
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
               o[4 * hh + 0] = __uint_as_float(acc[8 * u + 4 * hh + 0]) + bv.x;
               o[4 * hh + 1] = __uint_as_float(acc[8 * u + 4 * hh + 1]) + bv.y;
               o[4 * hh + 2] = __uint_as_float(acc[8 * u + 4 * hh + 2]) + bv.z;
@@ -724,18 +731,34 @@ TileChoice pick_tile(int M, int N, int G, int epi) {
   return {64, 1};
 }
 
+// Number of k slices gemm_tc will really use when `want` are asked for (slices hold whole
+// 64-deep k blocks, so the count can come out smaller).
+int gemm_tc_splits(int K, int want) {
+  if (want <= 1) return 1;
+  const int64_t nkb = ceil_div(K, BK);
+  return (int)ceil_div(nkb, ceil_div(nkb, want));
+}
+
 bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
   const int n_store = a.N_store > 0 ? a.N_store : a.N;
   const bool a_mn = a.a_sm == 1 && a.a_sk != 1, b_mn = a.b_sn == 1 && a.b_sk != 1;
   if (!a_mn && a.a_sk != 1) return false;
   if (!b_mn && a.b_sk != 1) return false;
-  const TileChoice tc = pick_tile(a.M, n_store, a.G, a.epi);
+  const TileChoice tc = pick_tile(a.M, n_store, a.G * (a.k_splits > 1 ? a.k_splits : 1), a.epi);
   const int bn = tc.bn, pair = tc.pair;
   TcArgs t{};
   t.M = a.M; t.N = n_store; t.K = a.K;
   t.m_tiles = (int)ceil_div(a.M, BM * pair);
   t.n_tiles = (int)ceil_div(n_store, bn);
   t.G = a.G;
+  t.k_splits = 1;
+  t.kb_per_split = (int)ceil_div(a.K, BK);
+  if (a.k_splits > 1) {
+    if (a.epi != EPI_BIAS_F32 || a.bias) return false;   // slices are plain fp32 partial products
+    t.kb_per_split = (int)ceil_div(ceil_div(a.K, BK), a.k_splits);
+    t.k_splits = (int)ceil_div(ceil_div(a.K, BK), t.kb_per_split);
+    if (t.k_splits != a.k_splits) return false;           // caller sizes its buffer with gemm_tc_splits()
+  }
   t.a_gmul = (a.G > 1 && a.a_sg != 0) ? 1 : 0;
   t.b_gmul = (a.G > 1 && a.b_sg != 0) ? 1 : 0;
   t.bias = a.bias; t.bias_sg = a.bias_sg;
@@ -762,8 +785,15 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
       if (bn == 128) return launch<0, 1, 128, 6, 0, 3, EPI_BIAS_RELU, 1>(L, m, t);
       return launch<0, 1, 64, 8, 0, 3, EPI_BIAS_RELU, 1>(L, m, t);
     case EPI_BIAS_F32:
-      if (a_mn || !b_mn) return false;
-      if (!make_map(&m.c32, a.outf, 4, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 128)) return false;
+      if (a_mn) return false;
+      if (!make_map(&m.c32, a.outf, 4, n_store, a.M, (long long)a.G * t.k_splits, a.outf_ld, a.outf_sg, CH, BM, 128))
+        return false;
+      if (!a_mn && !b_mn) {   // both operands K-major: k slices of delta * W^T
+        if (pair == 2) return launch<0, 0, 256, 6, 2, 0, EPI_BIAS_F32, 2>(L, m, t);
+        if (bn == 256) return launch<0, 0, 256, 4, 2, 0, EPI_BIAS_F32, 1>(L, m, t);
+        if (bn == 128) return launch<0, 0, 128, 5, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
+        return launch<0, 0, 64, 6, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
+      }
       if (pair == 2) return launch<0, 1, 256, 6, 2, 0, EPI_BIAS_F32, 2>(L, m, t);
       if (bn == 256) return launch<0, 1, 256, 4, 2, 0, EPI_BIAS_F32, 1>(L, m, t);
       if (bn == 128) return launch<0, 1, 128, 5, 3, 0, EPI_BIAS_F32, 1>(L, m, t);

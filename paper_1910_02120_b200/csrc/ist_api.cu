@@ -26,7 +26,7 @@ struct Region {
 // Placement of everything that lives in the caller's workspace blob.
 struct Plan {
   size_t total = 0;
-  Region status, part, row_loss, logits, ev_a, ev_b, ev_acc;
+  Region status, part, row_loss, logits, ev_a, ev_b, ev_acc, splitk;
   std::vector<Region> idx, off;             // hidden layer l at [l]  (1..t-1)
   std::vector<Region> master, bias, opw;    // layer l at [l]         (1..t)
   std::vector<Region> act, delta;           // act [0..t-1], delta [1..t]
@@ -132,6 +132,11 @@ bool valid_shape(const int64_t* dims, int n_dims, int S, int precision, int max_
   return true;
 }
 
+// delta_{l-1} = delta_l * W_l^T contracts over the width of layer l.  When that width is huge
+// (hundreds of thousands of classes) and the output small, the product has too few tiles to
+// fill the machine, so the contraction is cut into slices that run as separate tiles.
+int wanted_k_splits(int64_t K) { return K >= 16384 ? (int)std::min<int64_t>(64, ceil_div(K, 8192)) : 1; }
+
 void make_plan(ist_ctx* c) {
   Plan& p = c->plan;
   const int t = c->t, S = c->S;
@@ -163,6 +168,12 @@ void make_plan(ist_ctx* c) {
   p.ev_a = p.take((size_t)Bm * maxN * 4);
   p.ev_b = p.take((size_t)Bm * maxN * 4);
   p.ev_acc = p.take(64);
+  // fp32 partial products of k-split delta GEMMs (very wide layers only)
+  size_t sk = 0;
+  if (c->precision == IST_BF16)
+    for (int l = 2; l <= t; ++l)
+      sk = std::max(sk, (size_t)(wanted_k_splits(c->np[l]) > 1 ? wanted_k_splits(c->np[l]) : 0) * S * Bm * c->ld[l - 1] * 4);
+  p.splitk = p.take(sk);
 }
 
 void fill_shape(ist_ctx* c, const int64_t* dims, int n_dims, int S, int precision, int max_batch, int csr) {
@@ -257,6 +268,23 @@ bool gemm(ist_ctx* c, const GemmArgs<float>& a) {
   return true;
 }
 bool gemm(ist_ctx* c, const GemmArgs<bf16>& a) { return gemm_tc(c->launch(), a, c->status()); }
+
+// delta GEMM with the contraction cut into slices: fp32 partial slabs, then sum + ReLU mask.
+bool split_delta_gemm(ist_ctx*, const GemmArgs<float>&, int, int) { return false; }
+bool split_delta_gemm(ist_ctx* c, const GemmArgs<bf16>& masked, int want, int B) {
+  const int ks = gemm_tc_splits(masked.K, want);
+  float* part = c->plan.splitk.at<float>(c->ws);
+  GemmArgs<bf16> g = masked;
+  g.epi = EPI_BIAS_F32;
+  g.bias = nullptr;
+  g.k_splits = ks;
+  g.outf = part; g.outf_ld = masked.out_ld; g.outf_sg = (int64_t)B * masked.out_ld;
+  g.out = nullptr; g.mask = nullptr;
+  if (!gemm_tc(c->launch(), g, c->status())) return false;
+  splitk_mask_reduce<bf16>(c->launch(), part, ks, masked.G, B, masked.out_ld, masked.mask, masked.mask_sg, masked.out,
+                           masked.out_sg);
+  return true;
+}
 
 // One call of ist_local_steps in operand type T.
 template <typename T>
@@ -355,6 +383,10 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.mask = act(l - 1); g.mask_ld = c->ld[l - 1]; g.mask_sg = Bm * c->ld[l - 1];
         g.out = delta(l - 1); g.out_ld = c->ld[l - 1]; g.out_sg = Bm * c->ld[l - 1];
         Scope sc(c, IST_K_DX);
+        const int want = bf ? wanted_k_splits(c->np[l]) : 1;
+        if (want > 1) {
+          if (!split_delta_gemm(c, g, want, B)) return fail(c, IST_ERR_UNSUPPORTED, "k-split delta GEMM of layer %d cannot be launched", l);
+        } else
         if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMM of layer %d cannot be launched", l);
       }
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {

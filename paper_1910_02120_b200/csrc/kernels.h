@@ -68,6 +68,8 @@ template <typename T>
 struct GemmArgs {
   int M, N, K, G;
   int N_store;  // columns the epilogue may write (>= N, the padded row length); 0 = N
+  int k_splits; // > 1: cut the k range into this many slices; slice s of group g writes its fp32
+                // partial product to outf slab g * k_splits + s (EPI_BIAS_F32 without bias only)
   const T* A; int64_t a_sm, a_sk, a_sg;
   const T* B; int64_t b_sn, b_sk, b_sg;
   int epi;
@@ -82,6 +84,7 @@ template <typename T> void gemm_simt(const Launch& L, const GemmArgs<T>& a);
 // Tensor-core path (tcgen05 + TMA) for bf16 operands.  Returns false if the shape cannot be
 // described to TMA (misaligned strides) or the operand layouts do not fit an epilogue.
 bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st);
+int gemm_tc_splits(int K, int want);
 
 // ---- rowops.cu --------------------------------------------------------------------------
 // Row-wise softmax cross-entropy of logits [G][B][ld] against labels; writes
@@ -90,6 +93,11 @@ template <typename T>
 void softmax_xent(const Launch& L, const float* logits, int64_t ld, int64_t sg, int G, int B, int Nt,
                   const int32_t* y, int64_t y_sg, T* delta, int64_t ld_d, int64_t sg_d,
                   float* row_loss, DeviceStatus* st);
+// out[g][b][n] = T(mask[g][b][n] > 0 ? sum_s part[(g * ks + s)][b][n] : 0): closes a k-split
+// delta GEMM (fp32 partial slabs of B rows x ld columns each).
+template <typename T>
+void splitk_mask_reduce(const Launch& L, const float* part, int ks, int G, int B, int64_t ld, const T* mask,
+                        int64_t mask_sg, T* out, int64_t out_sg);
 // loss_out[g * out_stride + k] = (1/B) sum_b row_loss[g][b]  (fixed summation order)
 void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
                  int64_t out_stride, int k);

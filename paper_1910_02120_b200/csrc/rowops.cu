@@ -1,5 +1,7 @@
 // Row-wise pieces of a local SGD step that are not contractions: softmax cross-entropy and
 // its gradient, the bias update, input staging, and the evaluation reductions.
+#include <algorithm>
+
 #include "kernels.h"
 
 namespace ist {
@@ -67,6 +69,69 @@ __global__ void softmax_xent_kernel(const float* __restrict__ logits, int64_t ld
     d[n] = from_float<T>(v);
   }
   if (threadIdx.x == 0) row_loss[(int64_t)g * B + b] = logf(se) + mx - z[label];
+}
+
+// Wide rows (hundreds of thousands of classes): one pass with a running (max, sum) pair per
+// thread and 16-byte loads, then one pass that writes delta.  Row length ld is a multiple of 8.
+template <typename T>
+__global__ void __launch_bounds__(512) softmax_xent_wide_kernel(
+    const float* __restrict__ logits, int64_t ld, int64_t sg, int B, int Nt, const int32_t* __restrict__ y,
+    int64_t y_sg, T* __restrict__ delta, int64_t ld_d, int64_t sg_d, float* __restrict__ row_loss,
+    DeviceStatus* st) {
+  __shared__ float sm[16], ss[16];
+  pdl_wait();
+  pdl_trigger();
+  const int g = blockIdx.y, b = blockIdx.x;
+  const float* z = logits + (int64_t)g * sg + (int64_t)b * ld;
+  T* d = delta + (int64_t)g * sg_d + (int64_t)b * ld_d;
+  int label = y[(int64_t)g * y_sg + b];
+  if (label < 0 || label >= Nt) {
+    if (threadIdx.x == 0) report(st, -5, SITE_LABEL, (long long)g * B + b);
+    label = 0;
+  }
+  float m = -INFINITY, s = 0.f;
+  const int nvec = Nt / 4;
+  for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+    float4 t = *reinterpret_cast<const float4*>(z + 4 * v);
+    float mx = fmaxf(fmaxf(t.x, t.y), fmaxf(t.z, t.w));
+    if (mx > m) { s *= expf(m - mx); m = mx; }
+    s += expf(t.x - m) + expf(t.y - m) + expf(t.z - m) + expf(t.w - m);
+  }
+  for (int n = nvec * 4 + threadIdx.x; n < Nt; n += blockDim.x) {
+    float t = z[n];
+    if (t > m) { s *= expf(m - t); m = t; }
+    s += expf(t - m);
+  }
+  // combine (m, s) pairs: warp, then block
+  for (int o = 16; o; o >>= 1) {
+    float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+    float nm = fmaxf(m, om);
+    s = (m == -INFINITY ? 0.f : s * expf(m - nm)) + (om == -INFINITY ? 0.f : os * expf(om - nm));
+    m = nm;
+  }
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  if (l == 0) { sm[w] = m; ss[w] = s; }
+  __syncthreads();
+  float M = -INFINITY, S = 0.f;
+  for (int u = 0; u < (int)(blockDim.x >> 5); ++u) {   // fixed order, every thread the same
+    float nm = fmaxf(M, sm[u]);
+    S = (M == -INFINITY ? 0.f : S * expf(M - nm)) + (sm[u] == -INFINITY ? 0.f : ss[u] * expf(sm[u] - nm));
+    M = nm;
+  }
+  const float inv = 1.f / S, invB = 1.f / (float)B;
+  const int nvec_d = (int)(ld_d / 4);
+  for (int v = threadIdx.x; v < nvec_d; v += blockDim.x) {
+    float o[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int n = 4 * v + e;
+      o[e] = n < Nt ? (expf(z[n] - M) * inv - (n == label ? 1.f : 0.f)) * invB : 0.f;
+    }
+    T* dst = d + 4 * v;
+    dst[0] = from_float<T>(o[0]); dst[1] = from_float<T>(o[1]);
+    dst[2] = from_float<T>(o[2]); dst[3] = from_float<T>(o[3]);
+  }
+  if (threadIdx.x == 0) row_loss[(int64_t)g * B + b] = logf(S) + M - z[label];
 }
 
 __global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int B, float* loss_out,
@@ -196,6 +261,30 @@ __global__ void eval_finalize_kernel(const double* loss_sum, const long long* co
   *correct_out = (int64_t)*correct;
 }
 
+template <typename T>
+__global__ void splitk_mask_reduce_kernel(const float* __restrict__ part, int ks, int B, int64_t ld,
+                                          const T* __restrict__ mask, int64_t mask_sg, T* __restrict__ out,
+                                          int64_t out_sg) {
+  pdl_wait();
+  pdl_trigger();
+  const int g = blockIdx.y;
+  const int64_t per = (int64_t)B * ld;
+  for (int64_t e = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; e < per;
+       e += (int64_t)gridDim.x * blockDim.x * 4) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < ks; ++s) {   // fixed order
+      float4 v = *reinterpret_cast<const float4*>(part + ((int64_t)g * ks + s) * per + e);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    const T* m = mask + (int64_t)g * mask_sg + e;
+    T* o = out + (int64_t)g * out_sg + e;
+    o[0] = from_float<T>(to_float(m[0]) > 0.f ? acc.x : 0.f);
+    o[1] = from_float<T>(to_float(m[1]) > 0.f ? acc.y : 0.f);
+    o[2] = from_float<T>(to_float(m[2]) > 0.f ? acc.z : 0.f);
+    o[3] = from_float<T>(to_float(m[3]) > 0.f ? acc.w : 0.f);
+  }
+}
+
 int row_threads(int Nt) { return Nt <= 64 ? 32 : (Nt <= 1024 ? 128 : kThreads); }
 
 }  // namespace
@@ -204,8 +293,12 @@ template <typename T>
 void softmax_xent(const Launch& L, const float* logits, int64_t ld, int64_t sg, int G, int B, int Nt,
                   const int32_t* y, int64_t y_sg, T* delta, int64_t ld_d, int64_t sg_d,
                   float* row_loss, DeviceStatus* st) {
-  launch_pdl(softmax_xent_kernel<T>, dim3(B, G), dim3(row_threads(Nt)), 0, L.stream, logits, ld, sg, B, Nt, y, y_sg,
-             delta, ld_d, sg_d, row_loss, st);
+  if (Nt > 8192 && ld % 4 == 0 && ld_d % 4 == 0)
+    launch_pdl(softmax_xent_wide_kernel<T>, dim3(B, G), dim3(512), 0, L.stream, logits, ld, sg, B, Nt, y, y_sg, delta,
+               ld_d, sg_d, row_loss, st);
+  else
+    launch_pdl(softmax_xent_kernel<T>, dim3(B, G), dim3(row_threads(Nt)), 0, L.stream, logits, ld, sg, B, Nt, y, y_sg,
+               delta, ld_d, sg_d, row_loss, st);
   L.count();
 }
 template void softmax_xent<float>(const Launch&, const float*, int64_t, int64_t, int, int, int,
@@ -214,6 +307,17 @@ template void softmax_xent<float>(const Launch&, const float*, int64_t, int64_t,
 template void softmax_xent<bf16>(const Launch&, const float*, int64_t, int64_t, int, int, int,
                                  const int32_t*, int64_t, bf16*, int64_t, int64_t, float*,
                                  DeviceStatus*);
+
+template <typename T>
+void splitk_mask_reduce(const Launch& L, const float* part, int ks, int G, int B, int64_t ld, const T* mask,
+                        int64_t mask_sg, T* out, int64_t out_sg) {
+  const int64_t vecs = (int64_t)B * ld / 4;
+  dim3 grid((unsigned)std::min<int64_t>(ceil_div(vecs, 256), 1024), G);
+  launch_pdl(splitk_mask_reduce_kernel<T>, grid, dim3(256), 0, L.stream, part, ks, B, ld, mask, mask_sg, out, out_sg);
+  L.count();
+}
+template void splitk_mask_reduce<bf16>(const Launch&, const float*, int, int, int, int64_t, const bf16*, int64_t,
+                                       bf16*, int64_t);
 
 void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
                  int64_t out_stride, int k) {
