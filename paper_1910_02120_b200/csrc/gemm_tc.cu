@@ -689,7 +689,7 @@ bool launch(const Launch& L, const Maps& m, const TcArgs& t) {
       max_units = sm_count();
     }
   }
-  const int total = t.m_tiles * t.n_tiles * t.G;
+  const int total = t.m_tiles * t.n_tiles * t.G * t.k_splits;
   const int units = total < max_units ? total : max_units;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(PAIR * units);
@@ -794,6 +794,9 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
         if (bn == 128) return launch<0, 0, 128, 5, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
         return launch<0, 0, 64, 6, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
       }
+      // a short contraction (wide output layer fed by a narrow hidden layer) is bound by writing
+      // the logits: fewer operand stages, a deeper ring of output chunks
+      if (pair == 2 && ceil_div(a.K, BK) <= 4) return launch<0, 1, 256, 3, 6, 0, EPI_BIAS_F32, 2>(L, m, t);
       if (pair == 2) return launch<0, 1, 256, 6, 2, 0, EPI_BIAS_F32, 2>(L, m, t);
       if (bn == 256) return launch<0, 1, 256, 4, 2, 0, EPI_BIAS_F32, 1>(L, m, t);
       if (bn == 128) return launch<0, 1, 128, 5, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
