@@ -10,15 +10,18 @@
 //   warp 0 (one lane)  TMA loads of the A / B k-slabs into a ring of STAGES slots
 //   warp 1 (one lane)  tcgen05.mma issue; owns the tensor-memory allocation (2 accumulators,
 //                      so the MMAs of tile i+1 overlap the epilogue of tile i)
-//   warps 2..9         epilogue: tcgen05.ld (warp w reads lanes 32*(w%4)..+31, one row per
-//                      thread; the two warps of a lane quarter split a chunk's columns), 32
-//                      columns at a time, staged in swizzled shared memory and written with TMA
-//                      stores (coalesced, clipped at the tensor edge)
-//   warp 10 (one lane) TMA loads of the epilogue's input chunks: the fp32 master slice for the
-//                      SGD update, the ReLU mask for the delta GEMM
+//   warps 2..9         epilogue, two groups of four warps that take alternate 32-column chunks:
+//                      tcgen05.ld (warp w reads lanes 32*(w%4)..+31, one row per thread), apply
+//                      the epilogue, write the chunk into a swizzled shared-memory slot
+//   warp 10 (one lane) TMA loads of the epilogue's input chunks into the slots: the fp32 master
+//                      slice for the SGD update, the ReLU mask for the delta GEMM
+//   warp 11 (one lane) TMA stores of finished slots (coalesced, clipped at the tensor edge)
+// The epilogue has no CTA-wide barrier: slots move between loader, epilogue warps and storer
+// through mbarriers (slot_full -> chunk_done -> slot_empty), so warps work on different chunks
+// at the same time and a slow chunk does not hold the others back.
 // The weight-update epilogue is the HBM-heavy part of a step (10 bytes per weight against
-// 2*B flops): its fp32 master chunks are prefetched through a ring several chunks deep while
-// earlier chunks are updated in place in shared memory and stored back.
+// 2*B flops): its fp32 master chunks are prefetched through the slot ring while earlier chunks
+// are updated in place in shared memory and stored back.
 //
 // PAIR = 2 runs two CTAs of a cluster as one unit (tcgen05 cta_group::2): the pair computes a
 // 256 x BN tile, each CTA loads its own 128 rows of A and its half (BN/2 rows) of B and keeps its
@@ -47,8 +50,8 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;                   // 64 bf16 = 128 bytes = one swizzle row
 constexpr int CH = 32;                   // epilogue chunk: 32 output columns
-constexpr int kThreads = 352;
-constexpr int kEpiThreads = 256;
+constexpr int kThreads = 384;            // 12 warps, see the role list above
+constexpr int kEpiWarps = 8;
 constexpr int kAuxWarp = 10;
 constexpr long long kWaitLimitCycles = 2000000000ll;   // ~1 s at 2 GHz
 
@@ -139,21 +142,6 @@ __device__ __forceinline__ void tma_wait_read() {
 }
 __device__ __forceinline__ void tma_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
-// AND-reduction of a predicate over the epilogue threads, so that all of them leave together
-// when a bounded wait has expired for any of them.
-__device__ __forceinline__ bool epi_all(bool ok) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.b32 p, %1, 0;\n\t"
-      "bar.red.and.pred q, 2, %2, p;\n\t"
-      "selp.u32 %0, 1, 0, q;\n\t}"
-      : "=r"(r)
-      : "r"((uint32_t)ok), "n"(kEpiThreads)
-      : "memory");
-  return r != 0;
-}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
@@ -186,13 +174,16 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// 32 lanes x 16 consecutive 32-bit columns: thread i of the warp gets lane (row) i.
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t* v) {
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (row) i.
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* v) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -263,7 +254,7 @@ __device__ __forceinline__ uint4* b16_unit(uint8_t* area, int r, int u) {
   return reinterpret_cast<uint4*>(area + r * 64 + ((u ^ ((r >> 1) & 3)) << 4));
 }
 
-template <int A_MN, int B_MN, int BN, int STAGES, int N32, int N16, int EPI, int PAIR>
+template <int A_MN, int B_MN, int BN, int STAGES, int NS, int EPI, int PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC32,   // fp32 chunks: logits out, master in/out
@@ -271,24 +262,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmAux16, // bf16 chunks in: ReLU mask
                TcArgs a) {
   using ET = EpiTraits<EPI>;
-  static_assert(ET::k32 == (N32 > 0) && ET::k16 == (N16 > 0), "ring sizes do not match the epilogue");
   constexpr int BNL = BN / PAIR;   // rows of the B tile this CTA loads
   constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BNL * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-  constexpr uint32_t F32_BYTES = BM * CH * 4, B16_BYTES = BM * CH * 2;
-  constexpr int NAUX = EPI == EPI_SGD ? N32 : (EPI == EPI_RELU_MASK ? N16 : 1);
+  // a slot holds one 128 x 32 chunk: an fp32 area and / or a bf16 area, as the epilogue needs
+  constexpr uint32_t F32_BYTES = ET::k32 ? BM * CH * 4 : 0, B16_BYTES = ET::k16 ? BM * CH * 2 : 0;
+  constexpr uint32_t SLOT_BYTES = F32_BYTES + B16_BYTES;
   constexpr uint32_t AUX_BYTES = EPI == EPI_SGD ? F32_BYTES : B16_BYTES;
-  // Ring whose reuse only the storing thread gates (no loader refills it): the bf16 ring of the
-  // forward and update epilogues, the fp32 ring of the logits.  0 = every ring has a loader.
-  constexpr int NOUT = EPI == EPI_RELU_MASK ? 0 : (ET::k16 ? N16 : N32);
   constexpr uint32_t TMEM_COLS = 2 * BN;
   constexpr int NCH = BN / CH;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* ring32 = smem + STAGES * STAGE_BYTES;
-  uint8_t* ring16 = ring32 + N32 * F32_BYTES;
+  uint8_t* slots = smem + STAGES * STAGE_BYTES;
   __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
-  __shared__ uint64_t slot_full[NAUX], slot_empty[NAUX];
+  __shared__ uint64_t slot_full[NS], chunk_done[NS], slot_empty[NS];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
@@ -305,11 +292,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&acc_full[b], 1);
-      mbar_init(&acc_empty[b], PAIR * kEpiThreads / 32);   // one arrival per epilogue warp of the unit
+      mbar_init(&acc_empty[b], PAIR * kEpiWarps);   // one arrival per epilogue warp of the unit
     }
-    for (int s = 0; s < NAUX; ++s) {
-      mbar_init(&slot_full[s], 1);
-      mbar_init(&slot_empty[s], 1);
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(&slot_full[s], 1);               // loader's TMA bytes
+      mbar_init(&chunk_done[s], kEpiWarps / 2);  // the four warps that worked on the chunk
+      mbar_init(&slot_empty[s], 1);              // storer: the store has read the slot
     }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -445,37 +433,39 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp < kAuxWarp) {
     // ---------------------------------------------------------------- epilogue
     const int q = warp & 3;                           // tensor-memory lane quarter of this warp
-    const int h = (warp - 2) >> 2;                    // which 16 columns of a chunk
+    const int wg = (warp - 2) >> 2;                   // this warp's group takes chunks with cq % 2 == wg
     const int r = q * 32 + lane;                      // row of the tile owned by this thread
-    const bool leader = threadIdx.x == 64;            // issues the TMA stores
     int cq = 0, j = 0;
     bool ok = true;
     for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
-      const int m0 = (tile % a.m_tiles) * (BM * PAIR) + rank * BM;
       const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
-      const int g = tile / (a.m_tiles * a.n_tiles);
+      const int g = tile / (a.m_tiles * a.n_tiles);   // output slab (group, k slice)
       const int b = j & 1;
-      ok = epi_all(mbar_wait(&acc_full[b], (j >> 1) & 1, abortp, a.status, 4));
+      // warp-uniform outcome: the tensor-memory loads below need the whole warp
+      ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[b], (j >> 1) & 1, abortp, a.status, 4));
       if (!ok) break;
       tc_fence_after();
 #pragma unroll 1
       for (int c = 0; c < NCH; ++c, ++cq) {
         const int nc = n0 + c * CH;
         if (nc >= a.N) break;                         // CTA-uniform
-        uint8_t* f32 = ring32 + (N32 ? cq % (N32 ? N32 : 1) : 0) * F32_BYTES;
-        uint8_t* b16 = ring16 + (N16 ? cq % (N16 ? N16 : 1) : 0) * B16_BYTES;
-        if (ET::kAux) {
-          ok = epi_all(mbar_wait(&slot_full[cq % NAUX], (cq / NAUX) & 1, abortp, a.status, 5));
-          if (!ok) break;
-        }
-        uint32_t acc[16];
-        tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * CH + 16 * h), acc);
+        if ((cq & 1) != wg) continue;
+        const int slot = cq % NS;
+        uint8_t* f32 = slots + slot * SLOT_BYTES;
+        uint8_t* b16 = f32 + F32_BYTES;
+        // the slot is ready: loaded (input chunk) or drained by the store of an earlier chunk
+        if (ET::kAux) ok = mbar_wait(&slot_full[slot], (cq / NS) & 1, abortp, a.status, 5);
+        else ok = mbar_wait(&slot_empty[slot], ((cq / NS) & 1) ^ 1, abortp, a.status, 5);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        uint32_t acc[32];
+        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * CH), acc);
         if (EPI == EPI_SGD) {
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {               // 8 columns per iteration
+          for (int u = 0; u < 4; ++u) {               // 8 columns per iteration
             float w[8];
-            float4* p0 = f32_unit(f32, r, 4 * h + 2 * u);
-            float4* p1 = f32_unit(f32, r, 4 * h + 2 * u + 1);
+            float4* p0 = f32_unit(f32, r, 2 * u);
+            float4* p1 = f32_unit(f32, r, 2 * u + 1);
             float4 w0 = *p0, w1 = *p1;
             w[0] = w0.x - a.lr * __uint_as_float(acc[8 * u + 0]);
             w[1] = w0.y - a.lr * __uint_as_float(acc[8 * u + 1]);
@@ -487,13 +477,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             w[7] = w1.w - a.lr * __uint_as_float(acc[8 * u + 7]);
             *p0 = make_float4(w[0], w[1], w[2], w[3]);
             *p1 = make_float4(w[4], w[5], w[6], w[7]);
-            *b16_unit(b16, r, 2 * h + u) = pack8(w);
+            *b16_unit(b16, r, u) = pack8(w);
           }
         } else if (EPI == EPI_RELU_MASK) {
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {
+          for (int u = 0; u < 4; ++u) {
             float mk[8], o[8];
-            uint4* pm = b16_unit(b16, r, 2 * h + u);
+            uint4* pm = b16_unit(b16, r, u);
             unpack8(*pm, mk);
 #pragma unroll
             for (int e = 0; e < 8; ++e) o[e] = mk[e] > 0.f ? __uint_as_float(acc[8 * u + e]) : 0.f;
@@ -503,11 +493,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           // bias of the tile's group; a k slice of a split product carries none
           const float* bias = a.bias ? a.bias + (long long)(g / a.k_splits) * a.bias_sg : nullptr;
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {
+          for (int u = 0; u < 4; ++u) {
             float o[8];
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
-              const int n = nc + 16 * h + 8 * u + 4 * hh;
+              const int n = nc + 8 * u + 4 * hh;
               float4 bv = (bias && n < a.N) ? __ldg(reinterpret_cast<const float4*>(bias + n))
                                             : make_float4(0.f, 0.f, 0.f, 0.f);
               o[4 * hh + 0] = __uint_as_float(acc[8 * u + 4 * hh + 0]) + bv.x;
@@ -518,26 +508,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (EPI == EPI_BIAS_RELU) {
 #pragma unroll
               for (int e = 0; e < 8; ++e) o[e] = fmaxf(o[e], 0.f);
-              *b16_unit(b16, r, 2 * h + u) = pack8(o);
+              *b16_unit(b16, r, u) = pack8(o);
             } else {
-              *f32_unit(f32, r, 4 * h + 2 * u) = make_float4(o[0], o[1], o[2], o[3]);
-              *f32_unit(f32, r, 4 * h + 2 * u + 1) = make_float4(o[4], o[5], o[6], o[7]);
+              *f32_unit(f32, r, 2 * u) = make_float4(o[0], o[1], o[2], o[3]);
+              *f32_unit(f32, r, 2 * u + 1) = make_float4(o[4], o[5], o[6], o[7]);
             }
           }
         }
         fence_async_smem();          // generic-proxy writes -> visible to the TMA store
-        epi_barrier();
-        if (leader) {
-          if (ET::k32) tma_store_3d(&tmC32, f32, nc, m0, g);
-          if (ET::k16) tma_store_3d(&tmC16, b16, nc, m0, g);
-          tma_commit_group();
-          // The other threads run at most one chunk ahead of this one (they meet it again at
-          // the next barrier).  Letting one store stay in flight therefore keeps a ring of three
-          // areas safe; a ring of two must drain completely.
-          if (NOUT == 0 || NOUT >= 3) tma_wait_read<1>(); else tma_wait_read<0>();
-          // a loaded area may be refilled once the store that read it has finished with it
-          if (ET::kAux && cq >= 1) mbar_arrive(&slot_empty[(cq - 1) % NAUX]);
-        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&chunk_done[slot]);
       }
       if (!ok) break;
       tc_fence_before();
@@ -546,8 +526,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (PAIR == 2) mbar_arrive_cluster(map_to_cta(&acc_empty[b], 0)); else mbar_arrive(&acc_empty[b]);
       }
     }
-    if (leader) tma_wait_all();      // all stores complete before the CTA exits
-  } else {
+  } else if (warp == kAuxWarp) {
     // ---------------------------------------------------------------- epilogue input loads
     if (ET::kAux && lane == 0) {
       int cq = 0;
@@ -559,20 +538,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int c = 0; c < NCH; ++c, ++cq) {
           const int nc = n0 + c * CH;
           if (nc >= a.N) break;
-          const int slot = cq % NAUX;
-          ok = mbar_wait(&slot_empty[slot], ((cq / NAUX) & 1) ^ 1, abortp, a.status, 6);
+          const int slot = cq % NS;
+          ok = mbar_wait(&slot_empty[slot], ((cq / NS) & 1) ^ 1, abortp, a.status, 6);
           if (!ok) break;
           mbar_expect_tx(&slot_full[slot], AUX_BYTES);
-          if (EPI == EPI_SGD) tma_load_3d(ring32 + slot * F32_BYTES, &tmC32, &slot_full[slot], nc, m0, g);
-          else tma_load_3d(ring16 + slot * B16_BYTES, &tmAux16, &slot_full[slot], nc, m0, g);
+          if (EPI == EPI_SGD) tma_load_3d(slots + slot * SLOT_BYTES, &tmC32, &slot_full[slot], nc, m0, g);
+          else tma_load_3d(slots + slot * SLOT_BYTES + F32_BYTES, &tmAux16, &slot_full[slot], nc, m0, g);
         }
       }
       if (!ok) {
-        for (int jq = max(0, cq - NAUX); jq < cq; ++jq) {
+        for (int jq = max(0, cq - NS); jq < cq; ++jq) {
           long long t0 = clock64();
-          while (!mbar_try_wait(&slot_full[jq % NAUX], (jq / NAUX) & 1) && clock64() - t0 < kWaitLimitCycles) {}
+          while (!mbar_try_wait(&slot_full[jq % NS], (jq / NS) & 1) && clock64() - t0 < kWaitLimitCycles) {}
         }
       }
+    }
+  } else {
+    // ---------------------------------------------------------------- chunk stores
+    if (lane == 0) {
+      int cq = 0;
+      bool ok = true;
+      for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
+        const int m0 = (tile % a.m_tiles) * (BM * PAIR) + rank * BM;
+        const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
+        const int g = tile / (a.m_tiles * a.n_tiles);
+        for (int c = 0; c < NCH; ++c, ++cq) {
+          const int nc = n0 + c * CH;
+          if (nc >= a.N) break;
+          const int slot = cq % NS;
+          ok = mbar_wait(&chunk_done[slot], (cq / NS) & 1, abortp, a.status, 7);
+          if (!ok) break;
+          uint8_t* f32 = slots + slot * SLOT_BYTES;
+          if (ET::k32) tma_store_3d(&tmC32, f32, nc, m0, g);
+          if (ET::k16) tma_store_3d(&tmC16, f32 + F32_BYTES, nc, m0, g);
+          tma_commit_group();
+          // one store may stay in flight; the slot of the one before it has been read and can be
+          // refilled (by the loader) or rewritten (by the epilogue warps)
+          tma_wait_read<1>();
+          if (cq >= 1) mbar_arrive(&slot_empty[(cq - 1) % NS]);
+        }
+      }
+      tma_wait_all();                // all stores complete before the CTA exits
     }
   }
   tc_fence_before();
@@ -664,11 +670,13 @@ struct Maps {
   CUtensorMap a, b, c32, c16, aux16;
 };
 
-template <int A_MN, int B_MN, int BN, int STAGES, int N32, int N16, int EPI, int PAIR>
+template <int A_MN, int B_MN, int BN, int STAGES, int NS, int EPI, int PAIR>
 bool launch(const Launch& L, const Maps& m, const TcArgs& t) {
-  constexpr int smem = STAGES * (BM * BK * 2 + (BN / PAIR) * BK * 2) + N32 * BM * CH * 4 + N16 * BM * CH * 2 + 1024;
+  using ET = EpiTraits<EPI>;
+  constexpr int slot_bytes = (ET::k32 ? BM * CH * 4 : 0) + (ET::k16 ? BM * CH * 2 : 0);
+  constexpr int smem = STAGES * (BM * BK * 2 + (BN / PAIR) * BK * 2) + NS * slot_bytes + 1024;
   static_assert(smem <= 227 * 1024 - 512, "shared memory budget exceeded");
-  auto kern = gemm_tc_kernel<A_MN, B_MN, BN, STAGES, N32, N16, EPI, PAIR>;
+  auto kern = gemm_tc_kernel<A_MN, B_MN, BN, STAGES, NS, EPI, PAIR>;
   static int max_units = 0;   // CTAs (PAIR = 1) or clusters (PAIR = 2) that can be resident at once
   if (max_units == 0) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
@@ -780,42 +788,42 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
     case EPI_BIAS_RELU:
       if (a_mn || !b_mn) return false;
       if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
-      if (pair == 2) return launch<0, 1, 256, 6, 0, 3, EPI_BIAS_RELU, 2>(L, m, t);
-      if (bn == 256) return launch<0, 1, 256, 4, 0, 3, EPI_BIAS_RELU, 1>(L, m, t);
-      if (bn == 128) return launch<0, 1, 128, 6, 0, 3, EPI_BIAS_RELU, 1>(L, m, t);
-      return launch<0, 1, 64, 8, 0, 3, EPI_BIAS_RELU, 1>(L, m, t);
+      if (pair == 2) return launch<0, 1, 256, 6, 3, EPI_BIAS_RELU, 2>(L, m, t);
+      if (bn == 256) return launch<0, 1, 256, 4, 3, EPI_BIAS_RELU, 1>(L, m, t);
+      if (bn == 128) return launch<0, 1, 128, 6, 3, EPI_BIAS_RELU, 1>(L, m, t);
+      return launch<0, 1, 64, 8, 3, EPI_BIAS_RELU, 1>(L, m, t);
     case EPI_BIAS_F32:
       if (a_mn) return false;
       if (!make_map(&m.c32, a.outf, 4, n_store, a.M, (long long)a.G * t.k_splits, a.outf_ld, a.outf_sg, CH, BM, 128))
         return false;
       if (!a_mn && !b_mn) {   // both operands K-major: k slices of delta * W^T
-        if (pair == 2) return launch<0, 0, 256, 6, 2, 0, EPI_BIAS_F32, 2>(L, m, t);
-        if (bn == 256) return launch<0, 0, 256, 4, 2, 0, EPI_BIAS_F32, 1>(L, m, t);
-        if (bn == 128) return launch<0, 0, 128, 5, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
-        return launch<0, 0, 64, 6, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
+        if (pair == 2) return launch<0, 0, 256, 6, 2, EPI_BIAS_F32, 2>(L, m, t);
+        if (bn == 256) return launch<0, 0, 256, 4, 2, EPI_BIAS_F32, 1>(L, m, t);
+        if (bn == 128) return launch<0, 0, 128, 5, 3, EPI_BIAS_F32, 1>(L, m, t);
+        return launch<0, 0, 64, 6, 3, EPI_BIAS_F32, 1>(L, m, t);
       }
       // a short contraction (wide output layer fed by a narrow hidden layer) is bound by writing
       // the logits: fewer operand stages, a deeper ring of output chunks
-      if (pair == 2 && ceil_div(a.K, BK) <= 4) return launch<0, 1, 256, 3, 6, 0, EPI_BIAS_F32, 2>(L, m, t);
-      if (pair == 2) return launch<0, 1, 256, 6, 2, 0, EPI_BIAS_F32, 2>(L, m, t);
-      if (bn == 256) return launch<0, 1, 256, 4, 2, 0, EPI_BIAS_F32, 1>(L, m, t);
-      if (bn == 128) return launch<0, 1, 128, 5, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
-      return launch<0, 1, 64, 6, 3, 0, EPI_BIAS_F32, 1>(L, m, t);
+      if (pair == 2 && ceil_div(a.K, BK) <= 4) return launch<0, 1, 256, 3, 6, EPI_BIAS_F32, 2>(L, m, t);
+      if (pair == 2) return launch<0, 1, 256, 6, 2, EPI_BIAS_F32, 2>(L, m, t);
+      if (bn == 256) return launch<0, 1, 256, 4, 2, EPI_BIAS_F32, 1>(L, m, t);
+      if (bn == 128) return launch<0, 1, 128, 5, 3, EPI_BIAS_F32, 1>(L, m, t);
+      return launch<0, 1, 64, 6, 3, EPI_BIAS_F32, 1>(L, m, t);
     case EPI_RELU_MASK:
       if (a_mn || b_mn) return false;
       if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
       if (!make_map(&m.aux16, a.mask, 2, n_store, a.M, a.G, a.mask_ld, a.mask_sg, CH, BM, 64)) return false;
-      if (pair == 2) return launch<0, 0, 256, 6, 0, 4, EPI_RELU_MASK, 2>(L, m, t);
-      if (bn == 256) return launch<0, 0, 256, 4, 0, 4, EPI_RELU_MASK, 1>(L, m, t);
-      if (bn == 128) return launch<0, 0, 128, 6, 0, 4, EPI_RELU_MASK, 1>(L, m, t);
-      return launch<0, 0, 64, 8, 0, 4, EPI_RELU_MASK, 1>(L, m, t);
+      if (pair == 2) return launch<0, 0, 256, 6, 4, EPI_RELU_MASK, 2>(L, m, t);
+      if (bn == 256) return launch<0, 0, 256, 4, 4, EPI_RELU_MASK, 1>(L, m, t);
+      if (bn == 128) return launch<0, 0, 128, 6, 4, EPI_RELU_MASK, 1>(L, m, t);
+      return launch<0, 0, 64, 8, 4, EPI_RELU_MASK, 1>(L, m, t);
     case EPI_SGD:
       if (!a_mn || !b_mn || !a.opw) return false;
       if (!make_map(&m.c32, a.outf, 4, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 128)) return false;
       if (!make_map(&m.c16, a.opw, 2, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 64)) return false;
-      if (pair == 2) return launch<1, 1, 256, 4, 4, 3, EPI_SGD, 2>(L, m, t);
-      if (bn == 128) return launch<1, 1, 128, 4, 4, 3, EPI_SGD, 1>(L, m, t);
-      return launch<1, 1, 64, 5, 4, 3, EPI_SGD, 1>(L, m, t);
+      if (pair == 2) return launch<1, 1, 256, 4, 4, EPI_SGD, 2>(L, m, t);
+      if (bn == 128) return launch<1, 1, 128, 4, 4, EPI_SGD, 1>(L, m, t);
+      return launch<1, 1, 64, 5, 4, EPI_SGD, 1>(L, m, t);
     default:
       return false;
   }
