@@ -104,102 +104,176 @@ __device__ __forceinline__ void find_runs(const SliceMap& m, int S, int c0, int 
   __syncthreads();
 }
 
+// ---- bulk-copy helpers (one thread moves whole row segments asynchronously) -------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void bar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void bar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool bar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_addr(dst_smem)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, const void* src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+               ::"l"(dst), "r"(smem_addr(src_smem)), "r"(bytes) : "memory");
+}
+
+constexpr int kPermThreads = 512;
+constexpr long long kPermWaitCycles = 2000000000ll;   // ~1 s
+
+// Persistent CTA: column chunk blockIdx.x, row blocks blockIdx.y, blockIdx.y + gridDim.y, ...
+// The map from a packed position of the chunk to (column inside the chunk, offset in the packed
+// buffer) depends on the chunk only, so it is built once and reused for every row block.
+// Gather: row blocks arrive through double-buffered bulk copies (the next block loads while
+// this one is permuted).  Scatter: packed values are read into the permuted tile, which leaves
+// through bulk stores.  Requires full_cols % 4 == 0 (16-byte row segments).
 template <bool GATHER>
-__global__ void __launch_bounds__(256) permute_cols_kernel(float* __restrict__ W, SliceMap m, int S,
-                                                          float* __restrict__ master,
-                                                          bf16* __restrict__ opw) {
-  extern __shared__ float tile[];            // [kStageRows][kStageCols]
+__global__ void __launch_bounds__(kPermThreads, 1) permute_cols_kernel(float* __restrict__ W, SliceMap m, int S,
+                                                                      float* __restrict__ master,
+                                                                      bf16* __restrict__ opw, DeviceStatus* st) {
+  extern __shared__ __align__(128) unsigned char perm_smem[];
+  float* tile = reinterpret_cast<float*>(perm_smem);                                  // [2][rows][cols]
+  long long* map_off = reinterpret_cast<long long*>(tile + 2 * kStageRows * kStageCols);   // [cols]
+  uint16_t* map_col = reinterpret_cast<uint16_t*>(map_off + kStageCols);                   // [cols]
   __shared__ ColRuns runs;
+  __shared__ uint64_t full[2];
   const int c0 = blockIdx.x * kStageCols;
   const int c1 = min((int)m.full_cols, c0 + kStageCols);
   const int width = c1 - c0;
-  const int64_t k0 = (int64_t)blockIdx.y * kStageRows;
-  const int nrows = (int)min((long long)kStageRows, (long long)(m.full_rows - k0));
-  find_runs(m, S, c0, c1, &runs);
-
-  if (GATHER) {
-    // full matrix -> shared memory, coalesced (float4 where the row start allows it)
-    const bool vec = (m.full_cols % 4 == 0);
-    for (int r = 0; r < nrows; ++r) {
-      const float* src = W + (k0 + r) * m.full_cols + c0;
-      float* dst = tile + r * kStageCols;
-      if (vec) {
-        for (int v = threadIdx.x; v < width / 4; v += blockDim.x)
-          reinterpret_cast<float4*>(dst)[v] = __ldg(reinterpret_cast<const float4*>(src) + v);
-      } else {
-        for (int v = threadIdx.x; v < width; v += blockDim.x) dst[v] = __ldg(src + v);
-      }
-    }
-    __syncthreads();
+  const int64_t n_blocks = ceil_div(m.full_rows, kStageRows);
+  if (threadIdx.x == 0) {
+    bar_init(&full[0], 1);
+    bar_init(&full[1], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  // packed side: flattened over (group, position inside the run); one group's run is contiguous
+  find_runs(m, S, c0, c1, &runs);      // contains the barriers that publish the mbarrier init
   const int total = runs.pre[S];
-  for (int e = threadIdx.x; e < total; e += blockDim.x) {
+  for (int e = threadIdx.x; e < total; e += kPermThreads) {
     int s = 0;
     while (e >= runs.pre[s + 1]) ++s;
     const int j = runs.lo[s] + (e - runs.pre[s]);
-    const int col = m.col_idx[m.col_off[s] + j] - c0;
-    const int64_t o = ((int64_t)s * m.rows_pad + k0) * m.ld + j;
+    map_col[e] = (uint16_t)(m.col_idx[m.col_off[s] + j] - c0);
+    map_off[e] = (long long)s * m.rows_pad * m.ld + j;
+  }
+  __syncthreads();
+
+  auto issue_load = [&](int64_t rb, int buf) {   // thread 0 only
+    const int64_t k0 = rb * kStageRows;
+    const int nrows = (int)min((long long)kStageRows, (long long)(m.full_rows - k0));
+    bar_expect_tx(&full[buf], (uint32_t)(nrows * width * 4));
+    for (int r = 0; r < nrows; ++r)
+      bulk_load(tile + (buf * kStageRows + r) * kStageCols, W + (k0 + r) * m.full_cols + c0, (uint32_t)(width * 4),
+                &full[buf]);
+  };
+
+  if (GATHER && threadIdx.x == 0 && blockIdx.y < n_blocks) issue_load(blockIdx.y, 0);
+  int it = 0;
+  for (int64_t rb = blockIdx.y; rb < n_blocks; rb += gridDim.y, ++it) {
+    const int buf = it & 1;
+    const int64_t k0 = rb * kStageRows;
+    const int nrows = (int)min((long long)kStageRows, (long long)(m.full_rows - k0));
+    float* t = tile + buf * kStageRows * kStageCols;
     if (GATHER) {
+      // the other buffer was last read in the previous iteration, which ended with a barrier
+      if (threadIdx.x == 0 && rb + gridDim.y < n_blocks) issue_load(rb + gridDim.y, buf ^ 1);
+      bool ok = true;
+      const long long t0 = clock64();
+      while (!bar_try_wait(&full[buf], (it >> 1) & 1)) {
+        if (clock64() - t0 > kPermWaitCycles) { ok = false; break; }
+      }
+      if (!__syncthreads_and(ok)) {
+        if (threadIdx.x == 0) report(st, -6, SITE_TC_PIPE, 100);
+        return;
+      }
+      for (int e = threadIdx.x; e < total; e += kPermThreads) {
+        const int col = map_col[e];
+        const long long o = map_off[e] + k0 * m.ld;
 #pragma unroll
-      for (int r = 0; r < kStageRows; ++r) {
-        if (r < nrows) {
-          const float v = tile[r * kStageCols + col];
-          master[o + (int64_t)r * m.ld] = v;
-          if (opw) opw[o + (int64_t)r * m.ld] = __float2bfloat16_rn(v);
+        for (int r = 0; r < kStageRows; ++r) {
+          if (r < nrows) {
+            const float v = t[r * kStageCols + col];
+            master[o + (long long)r * m.ld] = v;
+            if (opw) opw[o + (long long)r * m.ld] = __float2bfloat16_rn(v);
+          }
         }
       }
+      if (blockIdx.x == 0) {   // pad columns [|G^s|, ld) of these rows are zero
+        for (int s = 0; s < S; ++s) {
+          const int cnt = m.col_off[s + 1] - m.col_off[s];
+          const int npad = (int)m.ld - cnt;
+          for (int e = threadIdx.x; e < npad * nrows; e += kPermThreads) {
+            const long long o = ((long long)s * m.rows_pad + k0 + e / npad) * m.ld + cnt + e % npad;
+            master[o] = 0.f;
+            if (opw) opw[o] = __float2bfloat16_rn(0.f);
+          }
+        }
+      }
+      __syncthreads();
     } else {
+      // this buffer's previous stores (two iterations ago) must have read it
+      if (threadIdx.x == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      __syncthreads();
+      for (int e = threadIdx.x; e < total; e += kPermThreads) {
+        const int col = map_col[e];
+        const long long o = map_off[e] + k0 * m.ld;
+        float v[kStageRows];
 #pragma unroll
-      for (int r = 0; r < kStageRows; ++r)
-        if (r < nrows) tile[r * kStageCols + col] = master[o + (int64_t)r * m.ld];
-    }
-  }
-  if (GATHER) {
-    // pad columns [|G^s|, ld) of these rows are zero (first column chunk does it)
-    if (blockIdx.x == 0) {
-      for (int s = 0; s < S; ++s) {
-        const int cnt = m.col_off[s + 1] - m.col_off[s];
-        const int npad = (int)m.ld - cnt;
-        for (int e = threadIdx.x; e < npad * nrows; e += blockDim.x) {
-          const int64_t o = ((int64_t)s * m.rows_pad + k0 + e / npad) * m.ld + cnt + e % npad;
-          master[o] = 0.f;
-          if (opw) opw[o] = __float2bfloat16_rn(0.f);
-        }
+        for (int r = 0; r < kStageRows; ++r) v[r] = r < nrows ? master[o + (long long)r * m.ld] : 0.f;
+#pragma unroll
+        for (int r = 0; r < kStageRows; ++r) t[r * kStageCols + col] = v[r];
       }
-    }
-  } else {
-    __syncthreads();
-    const bool vec = (m.full_cols % 4 == 0);
-    for (int r = 0; r < nrows; ++r) {
-      float* dst = W + (k0 + r) * m.full_cols + c0;
-      const float* src = tile + r * kStageCols;
-      if (vec) {
-        for (int v = threadIdx.x; v < width / 4; v += blockDim.x)
-          reinterpret_cast<float4*>(dst)[v] = reinterpret_cast<const float4*>(src)[v];
-      } else {
-        for (int v = threadIdx.x; v < width; v += blockDim.x) dst[v] = src[v];
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        for (int r = 0; r < nrows; ++r)
+          bulk_store(W + (k0 + r) * m.full_cols + c0, t + r * kStageCols, (uint32_t)(width * 4));
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
     }
   }
+  if (!GATHER && threadIdx.x == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 bool staged_ok(const SliceMap& m, int S) {
   return !m.row_idx && m.col_idx && m.full_rows >= kStageRows && S <= kMaxGroupsStaged &&
-         m.full_cols >= 256 && ceil_div(m.full_rows, kStageRows) <= 65535;
+         m.full_cols >= 256 && m.full_cols % 4 == 0;
 }
 
 template <bool GATHER>
-void launch_permute_cols(const Launch& L, float* W, const SliceMap& m, int S, float* master, bf16* opw) {
-  constexpr int smem = kStageRows * kStageCols * (int)sizeof(float);
+bool launch_permute_cols(const Launch& L, float* W, const SliceMap& m, int S, float* master, bf16* opw,
+                         DeviceStatus* st) {
+  constexpr int smem = 2 * kStageRows * kStageCols * (int)sizeof(float) + kStageCols * 8 + kStageCols * 2;
   static bool configured = false;
   if (!configured) {
-    cudaFuncSetAttribute(permute_cols_kernel<GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (cudaFuncSetAttribute(permute_cols_kernel<GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+        cudaSuccess)
+      return false;
     configured = true;
   }
-  dim3 grid((unsigned)ceil_div(m.full_cols, kStageCols), (unsigned)ceil_div(m.full_rows, kStageRows));
-  permute_cols_kernel<GATHER><<<grid, 256, smem, L.stream>>>(W, m, S, master, opw);
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int64_t chunks = ceil_div(m.full_cols, kStageCols), blocks = ceil_div(m.full_rows, kStageRows);
+  int64_t y = sms / chunks;
+  if (y < 1) y = 1;
+  if (y > blocks) y = blocks;
+  if (y > 65535) y = 65535;
+  dim3 grid((unsigned)chunks, (unsigned)y);
+  permute_cols_kernel<GATHER><<<grid, kPermThreads, smem, L.stream>>>(W, m, S, master, opw, st);
   L.count();
+  return true;
 }
 
 __global__ void mean_bias_kernel(float* b, int64_t n, int S, const float* __restrict__ packed,
@@ -223,21 +297,16 @@ __global__ void copy_out_kernel(const float* __restrict__ packed, int64_t ld, in
 }  // namespace
 
 void gather_slices(const Launch& L, const float* W, const SliceMap& m, int S, float* master,
-                   bf16* opw) {
-  if (staged_ok(m, S)) {
-    launch_permute_cols<true>(L, const_cast<float*>(W), m, S, master, opw);
-    return;
-  }
+                   bf16* opw, DeviceStatus* st) {
+  if (staged_ok(m, S) && launch_permute_cols<true>(L, const_cast<float*>(W), m, S, master, opw, st)) return;
   dim3 grid((unsigned)ceil_div(m.ld, kThreads), (unsigned)ceil_div(m.rows_pad, kRowsPerCta), S);
   gather_kernel<<<grid, kThreads, 0, L.stream>>>(W, m, master, opw);
   L.count();
 }
 
-void scatter_slices(const Launch& L, float* W, const SliceMap& m, int S, const float* master) {
-  if (staged_ok(m, S)) {
-    launch_permute_cols<false>(L, W, m, S, const_cast<float*>(master), nullptr);
-    return;
-  }
+void scatter_slices(const Launch& L, float* W, const SliceMap& m, int S, const float* master,
+                    DeviceStatus* st) {
+  if (staged_ok(m, S) && launch_permute_cols<false>(L, W, m, S, const_cast<float*>(master), nullptr, st)) return;
   dim3 grid((unsigned)ceil_div(m.ld, kThreads), (unsigned)ceil_div(m.rows_pad, kRowsPerCta), S);
   scatter_kernel<<<grid, kThreads, 0, L.stream>>>(W, m, master);
   L.count();

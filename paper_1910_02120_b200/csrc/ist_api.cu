@@ -493,8 +493,8 @@ extern "C" ist_status ist_partition(ist_ctx* c, uint64_t seed) {
   }
   for (int l = 1; l <= t; ++l) {
     Scope sc(c, IST_K_GATHER);
-    gather_slices(L, c->W[l - 1], slice_map(c, l), S, c->master(l), c->opw(l));
-    gather_slices(L, c->b[l - 1], bias_map(c, l), S, c->bias(l), nullptr);
+    gather_slices(L, c->W[l - 1], slice_map(c, l), S, c->master(l), c->opw(l), c->status());
+    gather_slices(L, c->b[l - 1], bias_map(c, l), S, c->bias(l), nullptr, c->status());
   }
   IST_CUDA(c, cudaGetLastError());
   c->state = ST_PARTITIONED;
@@ -553,8 +553,8 @@ extern "C" ist_status ist_reassemble(ist_ctx* c) {
   const int t = c->t, S = c->S;
   for (int l = 1; l <= t; ++l) {
     Scope sc(c, IST_K_SCATTER);
-    scatter_slices(L, c->W[l - 1], slice_map(c, l), S, c->master(l));
-    if (l < t) scatter_slices(L, c->b[l - 1], bias_map(c, l), S, c->bias(l));
+    scatter_slices(L, c->W[l - 1], slice_map(c, l), S, c->master(l), c->status());
+    if (l < t) scatter_slices(L, c->b[l - 1], bias_map(c, l), S, c->bias(l), c->status());
   }
   {
     Scope sc(c, IST_K_SCATTER);

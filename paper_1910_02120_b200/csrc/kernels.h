@@ -45,8 +45,9 @@ struct SliceMap {
   int64_t rows_pad, ld;          // packed slice: [S][rows_pad][ld]
 };
 void gather_slices(const Launch& L, const float* W, const SliceMap& m, int S, float* master,
-                   bf16* opw);
-void scatter_slices(const Launch& L, float* W, const SliceMap& m, int S, const float* master);
+                   bf16* opw, DeviceStatus* st);
+void scatter_slices(const Launch& L, float* W, const SliceMap& m, int S, const float* master,
+                    DeviceStatus* st);
 // b[j] += (sum_s (packed[s][j] - b[j])) / S for the output bias.
 void scatter_mean_bias(const Launch& L, float* b, int64_t n, int S, const float* packed,
                        int64_t ld);
