@@ -180,6 +180,34 @@ def test_csr_round(precision):
         _check_round(w, BF16_W_RTOL, BF16_DW_RTOL, BF16_LOSS_ATOL, False)
 
 
+def test_csr_rows_may_be_empty():
+    # a sample without features contributes only through the biases
+    import torch
+    from oracle import ist_oracle as O
+    dims, S, B, K = (50, 16, 6), 2, 4, 2
+    w = synth.Workload("e", dims, S=S, B=B, K=K, rounds=1, precision="fp32", x_dist="csr", lr=0.1, seed=3)
+    W, b = synth.make_weights(dims, 3, bias_scale=0.3)
+    rows = S * K * B
+    counts = np.array([0, 3, 0, 1] * (rows // 4))
+    rp = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    rng = np.random.default_rng(0)
+    col = np.concatenate([np.sort(rng.choice(dims[0], c, replace=False)) for c in counts]).astype(np.int32)
+    val = rng.random(col.size).astype(np.float32) + 0.5
+    y = synth.make_labels((S, K, B), dims[-1], 3)
+    o = O.IstOracle(dims, S)
+    o.bind_weights(W, b)
+    ol = o.round(9, (rp, col, val), y, w.lr, K)
+    ctx, Wd, bd = H.gpu_context(w, W, b)
+    X = (torch.tensor(rp, dtype=torch.int32, device="cuda:0"), torch.tensor(col, device="cuda:0"),
+         torch.tensor(val, device="cuda:0"))
+    gl = ctx.round(9, X, torch.tensor(y.reshape(-1), device="cuda:0"), w.lr, K, B).cpu().numpy()
+    ctx.sync_status()
+    np.testing.assert_allclose(gl, ol, rtol=1e-4)
+    for l in range(2):
+        H.assert_close(Wd[l].cpu().numpy(), o.W[l], FP32_RTOL)
+        H.assert_close(bd[l].cpu().numpy(), o.b[l], FP32_RTOL)
+
+
 def test_strides_zero_reuse_the_same_rows():
     # stride_step = 0 and stride_subnet = 0: every subnet and step sees batch 0
     import torch
