@@ -132,6 +132,15 @@ bool valid_shape(const int64_t* dims, int n_dims, int S, int precision, int max_
   return true;
 }
 
+// A narrow output layer (bf16 operands, at most 64 padded classes) is handled specially: its
+// logits GEMM is cut into k slices (more tiles, shorter pipelines) that the softmax kernel sums.
+constexpr int kHeadSplitsMax = 8;
+bool narrow_head(const ist_ctx* c) { return c->precision == IST_BF16 && c->t >= 2 && c->ld[c->t] <= 64; }
+int head_splits(const ist_ctx* c) {
+  const int64_t nkb = ceil_div(c->np[c->t - 1], 64);
+  return (int)std::max<int64_t>(1, std::min<int64_t>(kHeadSplitsMax, nkb / 4));
+}
+
 // delta_{l-1} = delta_l * W_l^T contracts over the width of layer l.  When that width is huge
 // (hundreds of thousands of classes) and the output small, the product has too few tiles to
 // fill the machine, so the contraction is cut into slices that run as separate tiles.
@@ -163,7 +172,7 @@ void make_plan(ist_ctx* c) {
   if (!c->csr) p.act[0] = p.take((size_t)S * Bm * c->ld[0] * es);   // staging of fp32 inputs
   for (int l = 1; l < t; ++l) p.act[l] = p.take((size_t)S * Bm * c->ld[l] * es);
   for (int l = 1; l <= t; ++l) p.delta[l] = p.take((size_t)S * Bm * c->ld[l] * es);
-  p.logits = p.take((size_t)S * Bm * c->ld[t] * 4);
+  p.logits = p.take((size_t)S * Bm * c->ld[t] * 4 * (narrow_head(c) ? kHeadSplitsMax : 1));
   p.row_loss = p.take((size_t)S * Bm * 4);
   p.ev_a = p.take((size_t)Bm * maxN * 4);
   p.ev_b = p.take((size_t)Bm * maxN * 4);
@@ -286,6 +295,16 @@ bool split_delta_gemm(ist_ctx* c, const GemmArgs<bf16>& masked, int want, int B)
   return true;
 }
 
+// Type-dispatch shims: the narrow-head kernels exist for bf16 operands only.
+int gemm_splits(int want, int K, const float*) { return 1; }
+int gemm_splits(int want, int K, const bf16*) { return gemm_tc_splits(K, want); }
+void small_softmax(const Launch&, const float*, int, int64_t, int, int, int, const float*, int64_t, const int32_t*,
+                   int64_t, float*, int64_t, int64_t, float*, DeviceStatus*) {}
+void small_softmax(const Launch& L, const float* part, int ks, int64_t ld, int G, int B, int Nt, const float* bias,
+                   int64_t bias_sg, const int32_t* y, int64_t y_sg, bf16* delta, int64_t ld_d, int64_t sg_d,
+                   float* row_loss, DeviceStatus* st) {
+  softmax_xent_small<bf16>(L, part, ks, ld, G, B, Nt, bias, bias_sg, y, y_sg, delta, ld_d, sg_d, row_loss, st);
+}
 // One call of ist_local_steps in operand type T.
 template <typename T>
 ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, float lr, int K,
@@ -327,6 +346,8 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
     auto in_ld = [&](int l) { return l == 0 ? a0_ld : c->ld[l]; };
     auto in_sg = [&](int l) { return l == 0 ? a0_sg : Bm * c->ld[l]; };
 
+    const bool head = narrow_head(c);
+    const int head_ks = head ? gemm_splits(head_splits(c), (int)c->np[t - 1], (const T*)nullptr) : 1;
     // ---- forward ---------------------------------------------------------------------------
     for (int l = 1; l <= t; ++l) {
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {
@@ -345,6 +366,11 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       if (l < t) {
         g.epi = EPI_BIAS_RELU;
         g.out = act(l); g.out_ld = c->ld[l]; g.out_sg = Bm * c->ld[l];
+      } else if (head) {
+        g.epi = EPI_BIAS_F32;        // k slices of the logits; bias and the sum happen in the softmax kernel
+        g.bias = nullptr;
+        g.k_splits = head_ks;
+        g.outf = logits; g.outf_ld = c->ld[t]; g.outf_sg = (int64_t)B * c->ld[t];
       } else {
         g.epi = EPI_BIAS_F32;
         g.outf = logits; g.outf_ld = c->ld[t]; g.outf_sg = Bm * c->ld[t];
@@ -355,6 +381,10 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
     // ---- loss and its gradient -------------------------------------------------------------
     {
       Scope sc(c, IST_K_LOSS);
+      if (head)
+        small_softmax(L, logits, head_ks, c->ld[t], S, B, (int)c->N[t], c->bias(t), c->ld[t], y + row0,
+                      X->stride_subnet, delta(t), c->ld[t], Bm * c->ld[t], row_loss, st);
+      else
       softmax_xent<T>(L, logits, c->ld[t], Bm * c->ld[t], S, B, (int)c->N[t], y + row0,
                       X->stride_subnet, delta(t), c->ld[t], Bm * c->ld[t], row_loss, st);
       if (loss_out) loss_reduce(L, row_loss, S, B, loss_out, K, k);
@@ -383,11 +413,13 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.mask = act(l - 1); g.mask_ld = c->ld[l - 1]; g.mask_sg = Bm * c->ld[l - 1];
         g.out = delta(l - 1); g.out_ld = c->ld[l - 1]; g.out_sg = Bm * c->ld[l - 1];
         Scope sc(c, IST_K_DX);
+        {
         const int want = bf ? wanted_k_splits(c->np[l]) : 1;
         if (want > 1) {
           if (!split_delta_gemm(c, g, want, B)) return fail(c, IST_ERR_UNSUPPORTED, "k-split delta GEMM of layer %d cannot be launched", l);
         } else
         if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMM of layer %d cannot be launched", l);
+        }
       }
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {
         Scope sc(c, IST_K_SPMM);

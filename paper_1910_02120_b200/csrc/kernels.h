@@ -99,6 +99,12 @@ void softmax_xent(const Launch& L, const float* logits, int64_t ld, int64_t sg, 
 template <typename T>
 void splitk_mask_reduce(const Launch& L, const float* part, int ks, int G, int B, int64_t ld, const T* mask,
                         int64_t mask_sg, T* out, int64_t out_sg);
+// Narrow output layer (Nt <= 64): softmax cross-entropy of logits given as ks partial slabs
+// ([G * ks][B][ld] fp32) plus bias; same outputs as softmax_xent.
+template <typename T>
+void softmax_xent_small(const Launch& L, const float* part, int ks, int64_t ld, int G, int B, int Nt,
+                        const float* bias, int64_t bias_sg, const int32_t* y, int64_t y_sg, T* delta, int64_t ld_d,
+                        int64_t sg_d, float* row_loss, DeviceStatus* st);
 // loss_out[g * out_stride + k] = (1/B) sum_b row_loss[g][b]  (fixed summation order)
 void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
                  int64_t out_stride, int k);

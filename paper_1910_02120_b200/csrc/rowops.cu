@@ -134,6 +134,52 @@ __global__ void __launch_bounds__(512) softmax_xent_wide_kernel(
   if (threadIdx.x == 0) row_loss[(int64_t)g * B + b] = logf(S) + M - z[label];
 }
 
+// Narrow output layer (Nt <= 64): one warp per row.  The logits may arrive as `ks` partial
+// products of a k-split GEMM (slab g * ks + s holds slice s of group g, B rows of ld columns);
+// they are summed here together with the bias, so the split costs no extra launch.
+template <typename T>
+__global__ void __launch_bounds__(256) softmax_xent_small_kernel(
+    const float* __restrict__ part, int ks, int64_t ld, int B, int Nt, const float* __restrict__ bias,
+    int64_t bias_sg, const int32_t* __restrict__ y, int64_t y_sg, T* __restrict__ delta, int64_t ld_d,
+    int64_t sg_d, float* __restrict__ row_loss, DeviceStatus* st) {
+  pdl_wait();
+  pdl_trigger();
+  const int g = blockIdx.y, lane = threadIdx.x & 31;
+  const int b = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (b >= B) return;
+  int label = y[(int64_t)g * y_sg + b];
+  if (label < 0 || label >= Nt) {
+    if (lane == 0) report(st, -5, SITE_LABEL, (long long)g * B + b);
+    label = 0;
+  }
+  float z[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int n = lane + 32 * h;
+    float v = -INFINITY;
+    if (n < Nt) {
+      v = bias ? bias[(int64_t)g * bias_sg + n] : 0.f;
+      for (int s = 0; s < ks; ++s) v += part[(((int64_t)g * ks + s) * B + b) * ld + n];   // fixed order
+    }
+    z[h] = v;
+  }
+  const float mx = warp_max(fmaxf(z[0], z[1]));
+  const float e0 = z[0] == -INFINITY ? 0.f : expf(z[0] - mx), e1 = z[1] == -INFINITY ? 0.f : expf(z[1] - mx);
+  const float se = warp_sum(e0 + e1);
+  const float zl = warp_sum((lane == (label & 31)) ? z[label >> 5] : 0.f);
+  const float inv = 1.f / se, invB = 1.f / (float)B;
+  T* d = delta + (int64_t)g * sg_d + (int64_t)b * ld_d;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int n = lane + 32 * h;
+    if (n < ld_d) {
+      const float e = h ? e1 : e0;
+      d[n] = from_float<T>(n < Nt ? (e * inv - (n == label ? 1.f : 0.f)) * invB : 0.f);
+    }
+  }
+  if (lane == 0) row_loss[(int64_t)g * B + b] = logf(se) + mx - zl;
+}
+
 __global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int B, float* loss_out,
                                    int64_t out_stride, int k) {
   __shared__ float sh[32];
@@ -318,6 +364,17 @@ void splitk_mask_reduce(const Launch& L, const float* part, int ks, int G, int B
 }
 template void splitk_mask_reduce<bf16>(const Launch&, const float*, int, int, int, int64_t, const bf16*, int64_t,
                                        bf16*, int64_t);
+
+template <typename T>
+void softmax_xent_small(const Launch& L, const float* part, int ks, int64_t ld, int G, int B, int Nt,
+                        const float* bias, int64_t bias_sg, const int32_t* y, int64_t y_sg, T* delta, int64_t ld_d,
+                        int64_t sg_d, float* row_loss, DeviceStatus* st) {
+  launch_pdl(softmax_xent_small_kernel<T>, dim3((unsigned)ceil_div(B, 8), G), dim3(256), 0, L.stream, part, ks, ld, B, Nt,
+             bias, bias_sg, y, y_sg, delta, ld_d, sg_d, row_loss, st);
+  L.count();
+}
+template void softmax_xent_small<bf16>(const Launch&, const float*, int, int64_t, int, int, int, const float*, int64_t,
+                                       const int32_t*, int64_t, bf16*, int64_t, int64_t, float*, DeviceStatus*);
 
 void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
                  int64_t out_stride, int k) {
