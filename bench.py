@@ -29,6 +29,10 @@ from paper_1910_02120_b200 import synth  # noqa: E402
 
 METRIC = "IST training samples/sec (all S subnets, device-timed)"
 UNIT = "samples/s"
+# DRAM bytes per algorithmic byte, from ncu captures of the named class's main launch
+# (profiles/gemm_tc_C3.md).  Valid for the kernels as they stand in this file's revision; set an
+# entry to None when the kernel changes.
+NCU_TRAFFIC_RATIO = {"C3-wide-pixels": {"dw_sgd": 488.9 / 503.3, "fwd": None, "dx": None}}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -42,6 +46,11 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--local-steps", type=int, default=0,
                     help="override K (local steps per round); makes a small case for profiler captures")
+    ap.add_argument("--sweep", action="store_true",
+                    help="run the scaling sweep (1024-H-H-100, batch 512, bf16) over H x S x K; one JSON line per point")
+    ap.add_argument("--sweep-H", default="2048,8192,32768,65536")
+    ap.add_argument("--sweep-S", default="1,2,4,8,16")
+    ap.add_argument("--sweep-K", default="1,10,100")
     ap.add_argument("--quick", action="store_true",
                     help="device-timed pass only (no end-to-end, per-class or CPU passes), warm-up as given")
     return ap.parse_args()
@@ -409,8 +418,10 @@ def run_ours(args, w):
     elif dominant in wm["bytes"] and (tensor_peak or dominant not in wm["flops"]):
         gbs = dk["gbs"]
         roof = {"kernel": dominant, "bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                "frac": gbs / pk["hbm_gbs"], "traffic": None, "peak_source": pk["_source"],
+                "frac": gbs / pk["hbm_gbs"], "peak_source": pk["_source"],
                 "bytes_per_launch": wm["bytes"][dominant] / dk["launches_per_step"],
+                "traffic": (NCU_TRAFFIC_RATIO.get(w.name, {}).get(dominant) or 0) * wm["bytes"][dominant] /
+                           dk["launches_per_step"] or None,
                 "avg_launch_ms": dk["ms_per_step"] / dk["launches_per_step"]}
     elif dominant in wm["flops"]:
         # fp32 CUDA-core contraction: 148 SMs x 128 FMA lanes x 2 flop x max clock
@@ -451,8 +462,66 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Scaling sweep: device-timed whole rounds at every (H, S, K); weights and inputs are drawn on
+    the device (same distributions as synth.py) so that the 17 GB networks need no host copy."""
+    import torch
+    from paper_1910_02120_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pk = peaks()
+    gen = torch.Generator(device=dev)
+    for H in [int(x) for x in args.sweep_H.split(",")]:
+        dims = (1024, H, H, 100)
+        gen.manual_seed(BASE_SWEEP_SEED + H)
+        Wd = []
+        for l in range(3):
+            bound = (6.0 / dims[l]) ** 0.5
+            Wd.append((torch.rand(dims[l], dims[l + 1], device=dev, generator=gen) * 2 - 1) * bound)
+        bd = [torch.zeros(dims[l + 1], device=dev) for l in range(3)]
+        for S in [int(x) for x in args.sweep_S.split(",")]:
+            ctx = api.Ist(dims, S, api.IST_BF16, 512, device=str(dev))
+            ctx.bind_weights(Wd, bd)
+            for K in [int(x) for x in args.sweep_K.split(",")]:
+                w = synth.c5(H, S, K)
+                X = torch.randn(S * K * 512, 1024, device=dev, generator=gen).to(torch.bfloat16)
+                y = torch.randint(0, 100, (S * K * 512,), device=dev, dtype=torch.int32, generator=gen)
+                loss = torch.empty(S * K, device=dev)
+                ctx.round(1, X, y, w.lr, K, 512, loss_out=loss)
+                ctx.sync_status()
+                reps = 3 if K >= 10 else 10
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for r in range(reps):
+                    ctx.round(2 + r, X, y, w.lr, K, 512, loss_out=loss)
+                e1.record()
+                torch.cuda.synchronize(dev)
+                ctx.sync_status()
+                ms = e0.elapsed_time(e1) / reps
+                wm = work_model(w)
+                flops = sum(wm["flops"].values())
+                print(json.dumps({"sweep": "C5", "H": H, "S": S, "K": K, "ms_per_round": ms,
+                                  "samples_per_s": w.samples_per_round / (ms * 1e-3),
+                                  "gemm_tflops_over_round": flops / (ms * 1e-3) / 1e12,
+                                  "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
+                                  "update_gbs_over_round": wm["bytes"]["dw_sgd"] / (ms * 1e-3) / 1e9,
+                                  "mean_loss": float(loss.mean().item())}), flush=True)
+                del X, y, loss
+            ctx.close()
+            del ctx
+            torch.cuda.empty_cache()
+        del Wd, bd
+        torch.cuda.empty_cache()
+
+
+BASE_SWEEP_SEED = 4321
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     w = synth.WORKLOADS[args.config]
     if args.local_steps > 0:
         w = w.scaled(K=args.local_steps, name=w.name + f"-K{args.local_steps}")
