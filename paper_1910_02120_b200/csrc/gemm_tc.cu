@@ -732,7 +732,7 @@ struct TileChoice { int bn, pair; };
 TileChoice pick_tile(int M, int N, int G, int epi) {
   const int sms = sm_count();
   auto tiles = [&](int bm, int bn) { return ceil_div(M, bm) * ceil_div(N, bn) * G; };
-  if (epi != EPI_SGD && M > BM && N > 128 && 4 * tiles(2 * BM, 256) >= 3 * (sms / 2)) return {256, 2};
+  if (M > BM && N > 128 && 4 * tiles(2 * BM, 256) >= 3 * (sms / 2)) return {256, 2};
   if (epi == EPI_SGD) return {(N > 64 && tiles(BM, 128) >= sms) ? 128 : 64, 1};
   if (N > 128 && tiles(BM, 256) >= sms) return {256, 1};
   if (N > 64 && tiles(BM, 128) >= sms) return {128, 1};
