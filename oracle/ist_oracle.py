@@ -23,7 +23,8 @@ What follows the paper, and what is a reading of it where the paper is silent:
   rows only.
 * App. A Eq. (2) with the n^2 factor removed, as Sec. 2.2 "Correcting
   Distributional Shift" does: f_l = S(W_l f_{l-1}) on the slice, scale 1.
-  READING: the batch standardisation of Sec. 2.2 is not applied here.
+  The batch standardisation of Sec. 2.2 is optional (`norm_eps`): off on the
+  plain path, on in the *_norm functions.
 * Sec. 2.1 "Training Subnets": J (= K here) iterations of local SGD per subnet,
   w <- w - eta * grad, no communication; then slices are copied back, with no
   collisions because the partition is disjoint.
@@ -262,9 +263,99 @@ def gradients(Ws, bs, X, y, dtype=np.float64):
     return loss, dW, db
 
 
-def sgd_step(Ws, bs, X, y, lr, dtype=np.float64):
+# ----------------------------------------------------------------------------
+# Sec. 2.2 "Correcting Distributional Shift": every hidden neuron's input is
+# standardised with the mean and standard deviation over the minibatch before
+# the non-linearity (no n^2 factor, no learned scale or shift).
+# READING: the paper gives no epsilon and does not say which variance; this
+# uses the biased (1/B) variance and sigma = sqrt(var + eps).
+# ----------------------------------------------------------------------------
+
+def forward_norm(Ws, bs, X, eps, dtype=np.float64):
+    """Forward pass with per-neuron batch standardisation in the hidden layers.
+
+    z_l = a_{l-1} W_l + b_l;  zh_l = (z_l - mean_b z_l) / sqrt(var_b z_l + eps);
+    a_l = max(zh_l, 0).  Returns z_t, the activations a_0..a_{t-1}, zh_1..zh_{t-1}
+    and 1/sigma_1..1/sigma_{t-1}.
+    """
+    t = len(Ws)
+    a = [X if isinstance(X, CsrRows) else np.asarray(X, dtype=dtype)]
+    zh, rstd = [], []
+    z = None
+    for l in range(1, t + 1):
+        prod = _first_layer_product(a[0], Ws[0], dtype) if l == 1 else a[l - 1] @ Ws[l - 1]
+        z = prod + bs[l - 1]
+        if l < t:
+            mu = z.mean(axis=0)
+            var = ((z - mu) ** 2).mean(axis=0)
+            r = 1.0 / np.sqrt(var + eps)
+            h = (z - mu) * r
+            zh.append(h)
+            rstd.append(r)
+            a.append(np.maximum(h, 0))
+    return z, a, zh, rstd
+
+
+def gradients_norm(Ws, bs, X, y, eps, dtype=np.float64):
+    """Loss and gradients with the standardisation differentiated through:
+    d_zh = (delta_{l+1} W_{l+1}^T) * [zh > 0];
+    d_z  = (d_zh - mean_b d_zh - zh * mean_b(d_zh * zh)) / sigma.
+    """
+    t = len(Ws)
+    z_t, a, zh, rstd = forward_norm(Ws, bs, X, eps, dtype)
+    loss, delta = softmax_xent(z_t, np.asarray(y, dtype=np.int64))
+    dW = [None] * t
+    db = [None] * t
+    for l in range(t, 0, -1):
+        db[l - 1] = delta.sum(axis=0)
+        if l == 1 and isinstance(X, CsrRows):
+            dW[0] = [(X.row(r)[0], np.outer(X.row(r)[1].astype(dtype), delta[r])) for r in range(X.B)]
+        else:
+            dW[l - 1] = a[l - 1].T @ delta
+        if l > 1:
+            h = zh[l - 2]
+            d_zh = (delta @ Ws[l - 1].T) * (h > 0)
+            delta = (d_zh - d_zh.mean(axis=0) - h * (d_zh * h).mean(axis=0)) * rstd[l - 2]
+    return loss, dW, db
+
+
+def calibrate(W, b, X, eps, dtype=np.float64):
+    """Deployment statistics (Sec. 2.2): mean and 1/sigma of every hidden neuron's input over a
+    data subset, computed with the full network layer by layer."""
+    _, _, zh, rstd = forward_norm(W, b, X, eps, dtype)
+    # forward_norm standardised with exactly these statistics; recover the means from it
+    stats = []
+    a = X if isinstance(X, CsrRows) else np.asarray(X, dtype=dtype)
+    for l in range(1, len(W)):
+        prod = _first_layer_product(a, W[0], dtype) if l == 1 else a @ W[l - 1]
+        z = prod + b[l - 1]
+        mu = z.mean(axis=0)
+        stats.append((mu, rstd[l - 1]))
+        a = np.maximum((z - mu) * rstd[l - 1], 0)
+    return stats
+
+
+def evaluate_norm(W, b, X, y, stats, dtype=np.float64):
+    """Full-width forward with stored statistics: mean loss and number of correct predictions."""
+    a = X if isinstance(X, CsrRows) else np.asarray(X, dtype=dtype)
+    t = len(W)
+    for l in range(1, t + 1):
+        prod = _first_layer_product(a, W[0], dtype) if l == 1 else a @ W[l - 1]
+        z = prod + b[l - 1]
+        if l < t:
+            mu, r = stats[l - 1]
+            a = np.maximum((z - mu) * r, 0)
+    y = np.asarray(y, dtype=np.int64)
+    loss, _ = softmax_xent(z, y)
+    return float(loss), int((z.argmax(axis=1) == y).sum())
+
+
+def sgd_step(Ws, bs, X, y, lr, dtype=np.float64, norm_eps=None):
     """One local SGD iteration, in place: w <- w - lr * grad.  Returns the pre-update loss."""
-    loss, dW, db = gradients(Ws, bs, X, y, dtype)
+    if norm_eps is None:
+        loss, dW, db = gradients(Ws, bs, X, y, dtype)
+    else:
+        loss, dW, db = gradients_norm(Ws, bs, X, y, norm_eps, dtype)
     lr = dtype(lr)
     for l in range(len(Ws)):
         if isinstance(dW[l], list):
@@ -292,7 +383,9 @@ def evaluate(W, b, X, y, dtype=np.float64):
 class IstOracle:
     """partition -> slice -> K local steps per subnet -> copy back."""
 
-    def __init__(self, layer_dims: Sequence[int], S: int, dtype=np.float64):
+    def __init__(self, layer_dims: Sequence[int], S: int, dtype=np.float64, norm_eps=None):
+        self.norm_eps = norm_eps          # None: plain path; a float: Sec. 2.2 standardisation
+        self.stats = None
         self.layer_dims = [int(d) for d in layer_dims]
         self.t = len(self.layer_dims) - 1
         if self.t < 1:
@@ -340,16 +433,24 @@ class IstOracle:
             Ws, bs = self.subnets[s]
             for k in range(K):
                 xb, yb = self._batch(X, y, s, k)
-                losses[s, k] = sgd_step(Ws, bs, xb, yb, lr, self.dtype)
+                losses[s, k] = sgd_step(Ws, bs, xb, yb, lr, self.dtype, self.norm_eps)
         return losses
 
     def reassemble(self):
         reassemble(self.W, self.b, self.parts, self.subnets)
         self.subnets = None
 
+    def calibrate(self, X):
+        if isinstance(X, tuple):
+            X = CsrRows(X[0], X[1], np.asarray(X[2], dtype=self.dtype))
+        self.stats = calibrate(self.W, self.b, X, self.norm_eps, self.dtype)
+        return self.stats
+
     def eval(self, X, y):
         if isinstance(X, tuple):
             X = CsrRows(X[0], X[1], np.asarray(X[2], dtype=self.dtype))
+        if self.norm_eps is not None:
+            return evaluate_norm(self.W, self.b, X, y, self.stats, self.dtype)
         return evaluate(self.W, self.b, X, y, self.dtype)
 
     def round(self, seed, X, y, lr, K):

@@ -387,3 +387,72 @@ def test_masked_linear_unbiased_scale_is_S_not_S_squared():
     err_S = np.linalg.norm(S * est - full) / np.linalg.norm(full)
     err_S2 = np.linalg.norm(S * S * est - full) / np.linalg.norm(full)
     assert err_S < 0.15 and err_S2 > 1.0
+
+
+# --- Sec. 2.2: per-neuron batch standardisation -------------------------------------------------
+
+def _torch_loss_norm(Ws, bs, X, y, eps):
+    a = X
+    for l in range(len(Ws)):
+        a = a @ Ws[l] + bs[l]
+        if l < len(Ws) - 1:
+            a = torch.nn.functional.batch_norm(a, None, None, training=True, eps=eps)   # no affine, batch stats
+            a = torch.relu(a)
+    return torch.nn.functional.cross_entropy(a, y, reduction="mean")
+
+
+@pytest.mark.parametrize("dims", [[6, 9, 4], [5, 8, 7, 3]])
+def test_norm_gradients_match_torch_batch_norm(dims):
+    eps = 1e-5
+    W, b, X, y = _tiny(dims, 1, 12, 1)
+    Ws = [w.astype(np.float64) for w in W]
+    bs = [v.astype(np.float64) for v in b]
+    loss, dW, db = O.gradients_norm(Ws, bs, X[0, 0].astype(np.float64), y[0, 0], eps)
+    tW = [torch.tensor(w, requires_grad=True) for w in Ws]
+    tb = [torch.tensor(v, requires_grad=True) for v in bs]
+    tl = _torch_loss_norm(tW, tb, torch.tensor(X[0, 0], dtype=torch.float64), torch.tensor(y[0, 0], dtype=torch.long), eps)
+    tl.backward()
+    assert abs(loss - tl.item()) < 1e-12
+    for l in range(len(Ws)):
+        np.testing.assert_allclose(dW[l], tW[l].grad.numpy(), rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(db[l], tb[l].grad.numpy(), rtol=1e-9, atol=1e-12)
+    # a hidden bias cancels in the standardisation: its gradient vanishes
+    for l in range(len(Ws) - 1):
+        assert np.max(np.abs(db[l])) < 1e-12
+
+
+def test_norm_forward_has_zero_mean_unit_variance():
+    dims = [7, 20, 15, 4]
+    W, b, X, _ = _tiny(dims, 1, 64, 1)
+    _, _, zh, _ = O.forward_norm([w.astype(np.float64) for w in W], [v.astype(np.float64) for v in b],
+                                 X[0, 0].astype(np.float64), 0.0)
+    for h in zh:
+        assert np.max(np.abs(h.mean(axis=0))) < 1e-12
+        np.testing.assert_allclose(h.var(axis=0), 1.0, rtol=1e-10)
+
+
+def test_norm_round_and_deployment_statistics():
+    # S = 1 round with standardisation equals torch SGD on the batch-normalised network, and
+    # evaluation with calibrated statistics equals the training-mode forward on the same rows
+    dims, B, K, lr, eps = [6, 10, 8, 4], 16, 3, 0.05, 1e-5
+    W, b, X, y = _tiny(dims, 1, B, K)
+    o = O.IstOracle(dims, 1, norm_eps=eps)
+    o.bind_weights(W, b)
+    losses = o.round(5, X, y, lr, K)
+    tW = [torch.tensor(w, dtype=torch.float64, requires_grad=True) for w in W]
+    tb = [torch.tensor(v, dtype=torch.float64, requires_grad=True) for v in b]
+    opt = torch.optim.SGD(tW + tb, lr=lr)
+    for k in range(K):
+        opt.zero_grad()
+        l = _torch_loss_norm(tW, tb, torch.tensor(X[0, k], dtype=torch.float64), torch.tensor(y[0, k], dtype=torch.long), eps)
+        l.backward()
+        opt.step()
+        assert abs(l.item() - losses[0, k]) < 1e-11
+    for l in range(3):
+        np.testing.assert_allclose(o.W[l], tW[l].detach().numpy(), rtol=1e-10, atol=1e-13)
+    o.calibrate(X[0, 0])
+    ev_loss, _ = o.eval(X[0, 0], y[0, 0])
+    with torch.no_grad():
+        ref = _torch_loss_norm([w.detach() for w in tW], [v.detach() for v in tb],
+                               torch.tensor(X[0, 0], dtype=torch.float64), torch.tensor(y[0, 0], dtype=torch.long), eps)
+    assert abs(ev_loss - ref.item()) < 1e-11
