@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C3", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--norm-eps", type=float, default=None,
+                    help="standardise hidden pre-activations over the batch (Sec. 2.2) with this epsilon")
     ap.add_argument("--local-steps", type=int, default=0,
                     help="override K (local steps per round); makes a small case for profiler captures")
     ap.add_argument("--sweep", action="store_true",
@@ -67,8 +69,10 @@ def peaks():
     return p
 
 
-def config_dict(w: synth.Workload, n_gpus: int):
+def config_dict(w: synth.Workload, n_gpus: int, norm_eps=None):
+    extra = {} if norm_eps is None else {"normalization": f"per-neuron batch standardisation, eps={norm_eps:g}"}
     return {
+        **extra,
         "workload": f"{w.name}: MLP {'-'.join(map(str, w.layer_dims))}, S={w.S}, batch={w.B}, "
                     f"K={w.K} local steps/round, {w.precision} operands, fp32 masters",
         "samples_per_step": w.samples_per_round,
@@ -83,7 +87,7 @@ def config_dict(w: synth.Workload, n_gpus: int):
 # algorithmic work per round (all S subnets), used for the roofline fractions
 # ---------------------------------------------------------------------------------------------
 
-def work_model(w: synth.Workload):
+def work_model(w: synth.Workload, norm=False):
     d, S, B, K = w.layer_dims, w.S, w.B, w.K
     t = len(d) - 1
     n = [d[0]] + [-(-d[l] // S) for l in range(1, t)] + [d[t]]
@@ -94,13 +98,17 @@ def work_model(w: synth.Workload):
     dx = 2 * B * S * sum(layer_elems[1:])
     dw = 2 * B * S * sum(layer_elems[(0 if dense_first else 1):])
     opw = 2 if w.precision == "bf16" else 0
+    es = 2 if w.precision == "bf16" else 4
+    hidden = B * S * sum(n[1:t])                    # hidden pre-activations per local step
+    # standardisation: forward reads fp32 z and writes a; backward reads z and d_zh, writes d_z
+    norm_bytes = {"norm": hidden * ((4 + es) + (4 + 2 * es)) * K} if norm else {}
     return {
         "packed_elems": packed,
         "flops": {"fwd": fwd * K, "dx": dx * K, "dw_sgd": dw * K},
         # bytes: gather = read fp32 + write fp32 master (+ bf16 copy); scatter = read + write fp32;
         # fused update inside dw_sgd = read + write master (+ bf16 copy)
         "bytes": {"gather": packed * (8 + opw), "scatter": packed * 8,
-                  "dw_sgd": packed * (8 + opw) * K},
+                  "dw_sgd": packed * (8 + opw) * K, **norm_bytes},
     }
 
 
@@ -175,11 +183,11 @@ class OracleSample:
     step on each of `n_sub` subnets, and the reassembly.  The round's throughput is extrapolated
     as S*K*B / (t_partition+slice+reassemble + S*K*t_step)."""
 
-    def __init__(self, w: synth.Workload, n_sub=1):
+    def __init__(self, w: synth.Workload, n_sub=1, norm_eps=None):
         from oracle import ist_oracle as O
-        self.O, self.w, self.n_sub = O, w, min(n_sub, w.S)
+        self.O, self.w, self.n_sub, self.norm_eps = O, w, min(n_sub, w.S), norm_eps
         W, b = synth.make_weights(w.layer_dims, w.seed)
-        self.o = O.IstOracle(w.layer_dims, w.S)
+        self.o = O.IstOracle(w.layer_dims, w.S, norm_eps=norm_eps)
         self.o.bind_weights(W, b)
         del W, b
         small = w.scaled(S=self.n_sub, K=1)
@@ -194,7 +202,7 @@ class OracleSample:
         for s in range(self.n_sub):
             Ws, bs = o.subnets[s]
             xb, yb = o._batch(X, self.data.y, s, 0)
-            self.O.sgd_step(Ws, bs, xb, yb, w.lr, o.dtype)
+            self.O.sgd_step(Ws, bs, xb, yb, w.lr, o.dtype, self.norm_eps)
         t2 = time.perf_counter()
         o.reassemble()
         t3 = time.perf_counter()
@@ -213,7 +221,7 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    smp = OracleSample(w)
+    smp = OracleSample(w, norm_eps=args.norm_eps)
     for i in range(args.warmup):
         smp.run(1000 + i)
     vals, secs = [], []
@@ -227,7 +235,7 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(secs)),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": config_dict(w, 1),
+        "data": "synthetic", "config": config_dict(w, 1, args.norm_eps),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": smp.describe()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -284,6 +292,8 @@ def run_ours(args, w):
     prec = api.IST_BF16 if w.precision == "bf16" else api.IST_FP32
     ctx = api.Ist(w.layer_dims, w.S, prec, w.B, input_is_csr=data.is_csr, device=str(dev))
     ctx.bind_weights(Wd, bd)
+    if args.norm_eps is not None:
+        ctx.enable_normalization(args.norm_eps)
     y_host = torch.from_numpy(data.y.reshape(-1).copy()).pin_memory()
     if data.is_csr:
         host_in = [torch.from_numpy(data.row_ptr.astype(np.int32)).pin_memory(),
@@ -335,7 +345,7 @@ def run_ours(args, w):
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                               "warmup": n_warm, "ms_per_step": ms / args.steps, "quick": True,
-                              "gpu_launches": launches, "config": config_dict(w, world)}))
+                              "gpu_launches": launches, "config": config_dict(w, world, args.norm_eps)}))
         if world > 1:
             dist.destroy_process_group()
         return
@@ -390,7 +400,7 @@ def run_ours(args, w):
         return
 
     pk = peaks()
-    wm = work_model(w)
+    wm = work_model(w, norm=args.norm_eps is not None)
     tensor_peak = pk["bf16_tflops_sustained"] if w.precision == "bf16" else None
     kernels = {}
     for name, (n, t_ms) in prof.items():
@@ -440,7 +450,7 @@ def run_ours(args, w):
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        smp = OracleSample(w, n_sub=2)
+        smp = OracleSample(w, n_sub=2, norm_eps=args.norm_eps)
         t0 = time.perf_counter()
         vals = []
         while len(vals) < 2 or (time.perf_counter() - t0 < 10 and len(vals) < 6):
@@ -452,7 +462,7 @@ def run_ours(args, w):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": n_warm, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.precision.replace("fp", "f"), "data": "synthetic",
-        "config": config_dict(w, world), "clocks": clocks,
+        "config": config_dict(w, world, args.norm_eps), "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": launches, "roofline": roof, "kernels": kernels, "cpu_baseline": cpu,

@@ -158,6 +158,32 @@ ist_status ist_reassemble(ist_ctx* ctx);
 ist_status ist_eval(ist_ctx* ctx, const ist_input* X, const int32_t* y_dev, int64_t n,
                     float* mean_loss_out_dev, int64_t* n_correct_out_dev);
 
+/*
+ * Sec. 2.2 "Correcting Distributional Shift", second remedy: every hidden neuron's input is
+ * standardised over the minibatch before the non-linearity,
+ *   zh = (z - mean_b z) / sqrt(var_b z + eps),  a = max(zh, 0),
+ * per subnet and neuron, with the biased (1/batch) variance and no learned scale or shift (the
+ * paper fixes neither eps nor the variance estimator), and the backward pass differentiates
+ * through it:  d_z = (d_zh - mean_b d_zh - zh * mean_b(d_zh * zh)) / sigma.
+ *
+ * ist_norm_workspace_bytes: bytes of a second device blob that holds the fp32 pre-activations
+ * of the hidden layers ([S][max_batch][n_l] per layer) and the statistics.
+ * ist_enable_normalization: switches the context to this mode for all later calls (there is no
+ * way back).  norm_workspace_dev: device, 256-byte aligned, at least that many bytes, borrowed
+ * until ist_destroy; it is cleared on the context's stream.  eps > 0.  Not allowed while a
+ * partition is in place.
+ * ist_calibrate: the deployment statistics of Sec. 2.2: mean and standard deviation of every
+ * hidden neuron's input over rows 0..n-1 of X (1 <= n <= max_batch, fp32 or CSR rows), computed
+ * with the bound full network layer by layer in fp32.  ist_eval then standardises with these
+ * stored values.  ist_reassemble and ist_bind_weights discard the statistics (they belong to the
+ * weights they were taken with); in this mode ist_eval without valid statistics returns
+ * IST_ERR_STATE.
+ */
+size_t ist_norm_workspace_bytes(const ist_ctx* ctx);
+ist_status ist_enable_normalization(ist_ctx* ctx, float eps, void* norm_workspace_dev,
+                                    size_t norm_workspace_bytes);
+ist_status ist_calibrate(ist_ctx* ctx, const ist_input* X, int64_t n);
+
 /* Waits for the stream and returns the sticky device status (IST_OK, IST_ERR_DEVICE_CHECK,
  * IST_ERR_DEVICE_TIMEOUT or IST_ERR_CUDA). */
 ist_status ist_sync_status(ist_ctx* ctx);
@@ -182,7 +208,8 @@ enum {
   IST_K_SPMM = 8,      /* sparse first layer: forward, backward + update */
   IST_K_SCATTER = 9,   /* packed slices -> full network */
   IST_K_EVAL = 10,     /* full-width evaluation */
-  IST_K_COUNT = 11
+  IST_K_NORM = 11,     /* batch standardisation, forward and backward (Sec. 2.2) */
+  IST_K_COUNT = 12
 };
 ist_status ist_profile(ist_ctx* ctx, int enable);
 ist_status ist_profile_read(ist_ctx* ctx, int kernel_class, int64_t* launches_out_host,

@@ -24,12 +24,12 @@ EXPORTS = [
     "ist_workspace_bytes", "ist_create", "ist_bind_weights", "ist_partition", "ist_get_partition",
     "ist_get_subnet_params", "ist_local_steps", "ist_reassemble", "ist_eval", "ist_sync_status",
     "ist_kernel_launches", "ist_last_error", "ist_destroy", "ist_profile", "ist_profile_read",
-    "ist_partition_layer_static",
+    "ist_partition_layer_static", "ist_norm_workspace_bytes", "ist_enable_normalization", "ist_calibrate",
 ]
 IST_STATIC_MAX_NEURONS, IST_STATIC_MAX_SUBNETS = 65536, 64
 
 KERNEL_CLASSES = ["partition", "gather", "stage", "fwd", "loss", "dx", "dw_sgd", "bias_sgd", "spmm",
-                  "scatter", "eval"]
+                  "scatter", "eval", "norm"]
 
 
 class IstInput(ctypes.Structure):
@@ -90,6 +90,12 @@ def _load() -> ctypes.CDLL:
     lib.ist_partition_layer_static.restype = ctypes.c_int32
     lib.ist_partition_layer_static.argtypes = [u64, i32, i64, i32, vp, vp, vp]
     lib.ist_destroy.restype = None
+    lib.ist_norm_workspace_bytes.argtypes = [vp]
+    lib.ist_norm_workspace_bytes.restype = sz
+    lib.ist_enable_normalization.argtypes = [vp, ctypes.c_float, vp, sz]
+    lib.ist_enable_normalization.restype = i32
+    lib.ist_calibrate.argtypes = [vp, ctypes.POINTER(IstInput), i64]
+    lib.ist_calibrate.restype = i32
     lib.ist_destroy.argtypes = [vp]
     return lib
 
@@ -259,6 +265,18 @@ class Ist:
         _check(self.handle, lib.ist_eval(self.handle, ctypes.byref(inp), y.data_ptr(), n,
                                          loss.data_ptr(), correct.data_ptr()))
         return loss, correct
+
+    def enable_normalization(self, eps: float):
+        """Sec. 2.2 batch standardisation of the hidden layers for all later calls."""
+        nbytes = int(lib.ist_norm_workspace_bytes(self.handle))
+        with torch.cuda.device(self.device):
+            self.norm_workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        _check(self.handle, lib.ist_enable_normalization(self.handle, ctypes.c_float(eps),
+                                                         self.norm_workspace.data_ptr(), nbytes))
+
+    def calibrate(self, X, n: int):
+        inp, keep = make_input(X, 0, 0, 0)
+        _check(self.handle, lib.ist_calibrate(self.handle, ctypes.byref(inp), n))
 
     def sync_status(self):
         _check(self.handle, lib.ist_sync_status(self.handle))

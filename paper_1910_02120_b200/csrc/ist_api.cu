@@ -38,6 +38,19 @@ struct Plan {
   }
 };
 
+// Placement of the buffers of the optional batch standardisation (a second caller-owned blob).
+struct NormPlan {
+  size_t total = 0;
+  std::vector<Region> z, mu, rstd;          // training: hidden layer l at [l], per subnet
+  std::vector<Region> ev_mu, ev_rstd;       // deployment statistics of the full network
+  Region take(size_t bytes) {
+    Region r;
+    r.offset = total;
+    total += (size_t)round_up((int64_t)bytes, 256);
+    return r;
+  }
+};
+
 }  // namespace
 
 struct ist_ctx {
@@ -53,6 +66,17 @@ struct ist_ctx {
   int64_t launches = 0;
   uint64_t seed = 0;
   std::string err;
+
+  // batch standardisation of hidden pre-activations (off unless ist_enable_normalization ran)
+  bool norm = false, calibrated = false;
+  float norm_eps = 0.f;
+  void* nws = nullptr;
+  NormPlan nplan;
+  float* zbuf(int l) const { return nplan.z[l].at<float>(nws); }
+  float* nmu(int l) const { return nplan.mu[l].at<float>(nws); }
+  float* nrstd(int l) const { return nplan.rstd[l].at<float>(nws); }
+  float* ev_mu(int l) const { return nplan.ev_mu[l].at<float>(nws); }
+  float* ev_rstd(int l) const { return nplan.ev_rstd[l].at<float>(nws); }
 
   // profiling: event pairs around groups of launches of one kernel class
   struct Span { int cls; int64_t kernels; cudaEvent_t a, b; };
@@ -185,6 +209,21 @@ void make_plan(ist_ctx* c) {
   p.splitk = p.take(sk);
 }
 
+void make_norm_plan(ist_ctx* c) {
+  NormPlan& p = c->nplan;
+  const int t = c->t;
+  p = NormPlan();
+  p.z.resize(t + 1); p.mu.resize(t + 1); p.rstd.resize(t + 1);
+  p.ev_mu.resize(t + 1); p.ev_rstd.resize(t + 1);
+  for (int l = 1; l < t; ++l) {
+    p.z[l] = p.take((size_t)c->S * c->max_batch * c->ld[l] * 4);
+    p.mu[l] = p.take((size_t)c->S * c->ld[l] * 4);
+    p.rstd[l] = p.take((size_t)c->S * c->ld[l] * 4);
+    p.ev_mu[l] = p.take((size_t)c->N[l] * 4);
+    p.ev_rstd[l] = p.take((size_t)c->N[l] * 4);
+  }
+}
+
 void fill_shape(ist_ctx* c, const int64_t* dims, int n_dims, int S, int precision, int max_batch, int csr) {
   c->t = n_dims - 1;
   c->S = S;
@@ -199,6 +238,7 @@ void fill_shape(ist_ctx* c, const int64_t* dims, int n_dims, int S, int precisio
     c->ld[l] = round_up(c->np[l], 8);
   }
   make_plan(c);
+  make_norm_plan(c);
 }
 
 ist_status cuda_fail(ist_ctx* c, cudaError_t e, const char* what) {
@@ -348,13 +388,27 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
 
     const bool head = narrow_head(c);
     const int head_ks = head ? gemm_splits(head_splits(c), (int)c->np[t - 1], (const T*)nullptr) : 1;
+    // Sec. 2.2: a_l = max((z_l - mean_b z_l) / sigma_b, 0) per subnet and neuron
+    auto standardise = [&](int l) {
+      Scope sc(c, IST_K_NORM);
+      colnorm_forward<T>(L, c->zbuf(l), c->ld[l], Bm * c->ld[l], S, B, (int)c->np[l], c->norm_eps, c->nmu(l),
+                         c->nrstd(l), c->ld[l], act(l), Bm * c->ld[l]);
+    };
     // ---- forward ---------------------------------------------------------------------------
     for (int l = 1; l <= t; ++l) {
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {
-        Scope sc(c, IST_K_SPMM);
-        spmm_forward<T, T>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
-                           weights(1), c->ld[1], c->slice_elems(1), c->bias(1), c->ld[1],
-                           (int)c->np[1], act(1), c->ld[1], Bm * c->ld[1], st);
+        {
+          Scope sc(c, IST_K_SPMM);
+          if (c->norm)
+            spmm_forward<T, float>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
+                                   weights(1), c->ld[1], c->slice_elems(1), c->bias(1), c->ld[1],
+                                   (int)c->np[1], c->zbuf(1), c->ld[1], Bm * c->ld[1], st, false);
+          else
+            spmm_forward<T, T>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
+                               weights(1), c->ld[1], c->slice_elems(1), c->bias(1), c->ld[1],
+                               (int)c->np[1], act(1), c->ld[1], Bm * c->ld[1], st);
+        }
+        if (c->norm) standardise(1);
         continue;
       }
       GemmArgs<T> g{};
@@ -363,7 +417,10 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       g.A = in_ptr(l - 1); g.a_sm = in_ld(l - 1); g.a_sk = 1; g.a_sg = in_sg(l - 1);
       g.B = weights(l); g.b_sn = 1; g.b_sk = c->ld[l]; g.b_sg = c->slice_elems(l);
       g.bias = c->bias(l); g.bias_sg = c->ld[l];
-      if (l < t) {
+      if (l < t && c->norm) {
+        g.epi = EPI_BIAS_F32;        // fp32 pre-activations; standardisation and ReLU follow
+        g.outf = c->zbuf(l); g.outf_ld = c->ld[l]; g.outf_sg = Bm * c->ld[l];
+      } else if (l < t) {
         g.epi = EPI_BIAS_RELU;
         g.out = act(l); g.out_ld = c->ld[l]; g.out_sg = Bm * c->ld[l];
       } else if (head) {
@@ -375,8 +432,11 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.epi = EPI_BIAS_F32;
         g.outf = logits; g.outf_ld = c->ld[t]; g.outf_sg = Bm * c->ld[t];
       }
-      Scope sc(c, IST_K_FWD);
-      if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "forward GEMM of layer %d cannot be launched", l);
+      {
+        Scope sc(c, IST_K_FWD);
+        if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "forward GEMM of layer %d cannot be launched", l);
+      }
+      if (l < t && c->norm) standardise(l);
     }
     // ---- loss and its gradient -------------------------------------------------------------
     {
@@ -420,6 +480,11 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         } else
         if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMM of layer %d cannot be launched", l);
         }
+      }
+      if (l > 1 && c->norm) {   // the masked product is d_zh; carry it through the standardisation
+        Scope sc(c, IST_K_NORM);
+        colnorm_backward<T>(L, delta(l - 1), c->ld[l - 1], Bm * c->ld[l - 1], c->zbuf(l - 1), Bm * c->ld[l - 1],
+                            c->nmu(l - 1), c->nrstd(l - 1), c->ld[l - 1], S, B, (int)c->np[l - 1]);
       }
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {
         Scope sc(c, IST_K_SPMM);
@@ -504,6 +569,7 @@ extern "C" ist_status ist_bind_weights(ist_ctx* c, float* const* W_dev, float* c
   }
   c->W.assign(W_dev, W_dev + c->t);
   c->b.assign(b_dev, b_dev + c->t);
+  c->calibrated = false;
   c->state = ST_BOUND;
   return IST_OK;
 }
@@ -594,55 +660,120 @@ extern "C" ist_status ist_reassemble(ist_ctx* c) {
   }
   IST_CUDA(c, cudaGetLastError());
   c->state = ST_BOUND;
+  c->calibrated = false;   // deployment statistics belong to the weights they were taken with
   return IST_OK;
 }
+
+namespace {
+
+// Full-width forward of rows r0..r0+rows-1 in fp32.  Hidden layers apply ReLU directly, or, in
+// normalisation mode, the stored statistics (measure = false) or statistics taken over these
+// very rows, which are then stored (measure = true).  Returns the buffer holding layer
+// `last`'s output (row stride N_last).
+const float* full_forward(ist_ctx* c, const ist_input* X, int64_t r0, int rows, int last, bool measure) {
+  Launch L = c->launch();
+  float* buf[2] = {c->plan.ev_a.at<float>(c->ws), c->plan.ev_b.at<float>(c->ws)};
+  const float* in = nullptr;
+  int64_t in_ld = 0;
+  int cur = 0;
+  for (int l = 1; l <= last; ++l) {
+    float* o = buf[cur];
+    const bool hidden = l < c->t;
+    if (l == 1 && X->kind == IST_X_CSR) {
+      spmm_forward<float, float>(L, X->row_ptr, X->col, X->val, r0, 0, 1, rows, c->N[0], c->W[0], c->N[1],
+                                 0, c->b[0], 0, (int)c->N[1], o, c->N[1], 0, c->status(), !c->norm);
+    } else {
+      GemmArgs<float> g{};
+      g.M = rows; g.N = (int)c->N[l]; g.K = (int)c->N[l - 1]; g.G = 1;
+      if (l == 1) { g.A = reinterpret_cast<const float*>(X->dense) + r0 * c->N[0]; g.a_sm = c->N[0]; }
+      else { g.A = in; g.a_sm = in_ld; }
+      g.a_sk = 1;
+      g.B = c->W[l - 1]; g.b_sn = 1; g.b_sk = c->N[l];
+      g.bias = c->b[l - 1];
+      if (hidden && !c->norm) { g.epi = EPI_BIAS_RELU; g.out = o; g.out_ld = c->N[l]; }
+      else { g.epi = EPI_BIAS_F32; g.outf = o; g.outf_ld = c->N[l]; }
+      gemm_simt<float>(L, g);
+    }
+    if (hidden && c->norm) {
+      if (measure)
+        colnorm_forward<float>(L, o, c->N[l], 0, 1, rows, (int)c->N[l], c->norm_eps, c->ev_mu(l), c->ev_rstd(l), 0,
+                               o, 0);
+      else
+        colnorm_apply(L, o, c->N[l], rows, (int)c->N[l], c->ev_mu(l), c->ev_rstd(l));
+    }
+    in = o;
+    in_ld = c->N[l];
+    cur ^= 1;
+  }
+  return in;
+}
+
+}  // namespace
 
 extern "C" ist_status ist_eval(ist_ctx* c, const ist_input* X, const int32_t* y_dev, int64_t n,
                                float* mean_loss_out_dev, int64_t* n_correct_out_dev) {
   if (!c) return IST_ERR_ARG;
   if (c->state != ST_BOUND) return fail(c, IST_ERR_STATE, "ist_eval needs bound weights and no partition in place");
+  if (c->norm && c->t > 1 && !c->calibrated)
+    return fail(c, IST_ERR_STATE, "normalisation is enabled: ist_calibrate must run before ist_eval");
   if (n < 1) return fail(c, IST_ERR_ARG, "n must be >= 1");
   if (!mean_loss_out_dev || !n_correct_out_dev) return fail(c, IST_ERR_ARG, "output pointers must not be null");
   ist_status s = check_input(c, X, y_dev, false);
   if (s != IST_OK) return s;
   if (X->kind == IST_X_DENSE_BF16) return fail(c, IST_ERR_UNSUPPORTED, "ist_eval takes fp32 or CSR rows");
   Launch L = c->launch();
-  const int t = c->t;
-  float* buf[2] = {c->plan.ev_a.at<float>(c->ws), c->plan.ev_b.at<float>(c->ws)};
   double* loss_sum = c->plan.ev_acc.at<double>(c->ws);
   long long* correct = reinterpret_cast<long long*>(loss_sum + 1);
   IST_CUDA(c, cudaMemsetAsync(loss_sum, 0, 16, c->stream));
   Scope sc(c, IST_K_EVAL);
   for (int64_t r0 = 0; r0 < n; r0 += c->max_batch) {
     const int rows = (int)std::min<int64_t>(c->max_batch, n - r0);
-    const float* in = nullptr;
-    int64_t in_ld = 0;
-    int cur = 0;
-    for (int l = 1; l <= t; ++l) {
-      float* o = buf[cur];
-      if (l == 1 && X->kind == IST_X_CSR) {
-        spmm_forward<float, float>(L, X->row_ptr, X->col, X->val, r0, 0, 1, rows, c->N[0], c->W[0], c->N[1],
-                                   0, c->b[0], 0, (int)c->N[1], o, c->N[1], 0, c->status());
-      } else {
-        GemmArgs<float> g{};
-        g.M = rows; g.N = (int)c->N[l]; g.K = (int)c->N[l - 1]; g.G = 1;
-        if (l == 1) { g.A = reinterpret_cast<const float*>(X->dense) + r0 * c->N[0]; g.a_sm = c->N[0]; }
-        else { g.A = in; g.a_sm = in_ld; }
-        g.a_sk = 1;
-        g.B = c->W[l - 1]; g.b_sn = 1; g.b_sk = c->N[l];
-        g.bias = c->b[l - 1];
-        if (l < t) { g.epi = EPI_BIAS_RELU; g.out = o; g.out_ld = c->N[l]; }
-        else { g.epi = EPI_BIAS_F32; g.outf = o; g.outf_ld = c->N[l]; }
-        gemm_simt<float>(L, g);
-      }
-      in = o;
-      in_ld = c->N[l];
-      cur ^= 1;
-    }
-    eval_rows(L, in, in_ld, rows, (int)c->N[t], y_dev + r0, loss_sum, correct, c->status());
+    const float* logits = full_forward(c, X, r0, rows, c->t, false);
+    eval_rows(L, logits, c->N[c->t], rows, (int)c->N[c->t], y_dev + r0, loss_sum, correct, c->status());
   }
   eval_finalize(L, loss_sum, correct, n, mean_loss_out_dev, n_correct_out_dev);
   IST_CUDA(c, cudaGetLastError());
+  return IST_OK;
+}
+
+extern "C" size_t ist_norm_workspace_bytes(const ist_ctx* c) { return c ? std::max<size_t>(c->nplan.total, 256) : 0; }
+
+extern "C" ist_status ist_enable_normalization(ist_ctx* c, float eps, void* norm_workspace_dev,
+                                               size_t norm_workspace_bytes) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state == ST_PARTITIONED)
+    return fail(c, IST_ERR_STATE, "normalisation cannot be switched on between ist_partition and ist_reassemble");
+  if (c->norm) return fail(c, IST_ERR_STATE, "normalisation is already enabled");
+  if (!(eps > 0.f) || !(eps < 1e30f)) return fail(c, IST_ERR_ARG, "eps must be a positive finite number");
+  if (!norm_workspace_dev || ((uintptr_t)norm_workspace_dev & 255))
+    return fail(c, IST_ERR_WORKSPACE, "normalisation workspace must be a 256-byte aligned device pointer");
+  if (norm_workspace_bytes < c->nplan.total)
+    return fail(c, IST_ERR_WORKSPACE, "normalisation workspace holds %zu bytes, %zu needed", norm_workspace_bytes,
+                c->nplan.total);
+  if (c->nplan.total) IST_CUDA(c, cudaMemsetAsync(norm_workspace_dev, 0, c->nplan.total, c->stream));
+  c->nws = norm_workspace_dev;
+  c->norm_eps = eps;
+  c->norm = true;
+  c->calibrated = false;
+  return IST_OK;
+}
+
+extern "C" ist_status ist_calibrate(ist_ctx* c, const ist_input* X, int64_t n) {
+  if (!c) return IST_ERR_ARG;
+  if (!c->norm) return fail(c, IST_ERR_STATE, "ist_calibrate needs ist_enable_normalization first");
+  if (c->state != ST_BOUND) return fail(c, IST_ERR_STATE, "ist_calibrate needs bound weights and no partition in place");
+  if (n < 1 || n > c->max_batch) return fail(c, IST_ERR_ARG, "n must be in 1..max_batch (%d)", c->max_batch);
+  if (!X) return fail(c, IST_ERR_ARG, "X must not be null");
+  const int32_t dummy = 0;
+  ist_status s = check_input(c, X, &dummy, false);
+  if (s != IST_OK) return s;
+  if (X->kind == IST_X_DENSE_BF16) return fail(c, IST_ERR_UNSUPPORTED, "ist_calibrate takes fp32 or CSR rows");
+  {
+    Scope sc(c, IST_K_EVAL);
+    full_forward(c, X, 0, (int)n, c->t - 1, true);
+  }
+  IST_CUDA(c, cudaGetLastError());
+  c->calibrated = true;
   return IST_OK;
 }
 

@@ -129,13 +129,24 @@ void eval_rows(const Launch& L, const float* logits, int64_t ld, int rows, int N
 void eval_finalize(const Launch& L, const double* loss_sum, const long long* correct, int64_t n,
                    float* mean_loss_out, int64_t* correct_out);
 
+// ---- colnorm.cu -------------------------------------------------------------------------
+// Batch standardisation of hidden pre-activations (Sec. 2.2).  z [G][B][ld] fp32, statistics
+// [G][ld] (stat_sg apart), act / delta [G][B][ld] in operand precision.  n live columns.
+template <typename T>
+void colnorm_forward(const Launch& L, const float* z, int64_t ld, int64_t z_sg, int G, int B, int n, float eps,
+                     float* mu, float* rstd, int64_t stat_sg, T* act, int64_t act_sg);
+template <typename T>
+void colnorm_backward(const Launch& L, T* delta, int64_t ld, int64_t d_sg, const float* z, int64_t z_sg, const float* mu,
+                      const float* rstd, int64_t stat_sg, int G, int B, int n);
+void colnorm_apply(const Launch& L, float* z, int64_t ld, int rows, int n, const float* mu, const float* rstd);
+
 // ---- spmm.cu ----------------------------------------------------------------------------
 // out[g][b][:] = relu(sum_nz val * P[g][col][:] + bias[g][:]) for rows r0_g + b of a CSR matrix.
 template <typename T, typename TO>
 void spmm_forward(const Launch& L, const int32_t* row_ptr, const int32_t* col, const float* val,
                   int64_t row0, int64_t group_row_stride, int G, int B, int64_t N0, const T* P,
                   int64_t p_ld, int64_t p_sg, const float* bias, int64_t bias_sg, int n1, TO* out,
-                  int64_t out_ld, int64_t out_sg, DeviceStatus* st);
+                  int64_t out_ld, int64_t out_sg, DeviceStatus* st, bool relu = true);
 // master[g][col][:] -= lr * val * delta[g][b][:] over stored nonzeros (atomic adds), then
 // refresh the bf16 copy of the touched rows (opw may be null).
 template <typename T>

@@ -12,27 +12,6 @@ namespace {
 
 constexpr int kRowsPerCta = 4;
 
-__device__ __forceinline__ void load4(const float* p, float v[4]) {
-  float4 t = *reinterpret_cast<const float4*>(p);
-  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-}
-__device__ __forceinline__ void load4(const bf16* p, float v[4]) {
-  uint2 t = *reinterpret_cast<const uint2*>(p);
-  __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&t.x);
-  __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&t.y);
-  v[0] = __low2float(a); v[1] = __high2float(a); v[2] = __low2float(b); v[3] = __high2float(b);
-}
-__device__ __forceinline__ void store4(float* p, const float v[4]) {
-  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
-}
-__device__ __forceinline__ void store4(bf16* p, const float v[4]) {
-  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
-  __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
-  uint2 t;
-  t.x = *reinterpret_cast<uint32_t*>(&a);
-  t.y = *reinterpret_cast<uint32_t*>(&b);
-  *reinterpret_cast<uint2*>(p) = t;
-}
 
 // VEC = false: element-wise accesses for leading dimensions that are not multiples of 4
 // (the full network's first layer during evaluation).
@@ -43,7 +22,7 @@ __global__ void spmm_forward_kernel(const int32_t* __restrict__ row_ptr, const i
                                     const T* __restrict__ P, int64_t p_ld, int64_t p_sg,
                                     const float* __restrict__ bias, int64_t bias_sg, int n1,
                                     TO* __restrict__ out, int64_t out_ld, int64_t out_sg,
-                                    DeviceStatus* st) {
+                                    DeviceStatus* st, bool relu) {
   int g = blockIdx.y;
   int b = blockIdx.x * kRowsPerCta + threadIdx.y;
   int cc = blockIdx.z * 128 + threadIdx.x * 4;
@@ -77,7 +56,7 @@ __global__ void spmm_forward_kernel(const int32_t* __restrict__ row_ptr, const i
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
     float bv = (cc + u) < n1 ? bias[(int64_t)g * bias_sg + cc + u] : 0.f;
-    o[u] = fmaxf(acc[u] + bv, 0.f);
+    o[u] = relu ? fmaxf(acc[u] + bv, 0.f) : acc[u] + bv;
   }
   TO* dst = out + (int64_t)g * out_sg + (int64_t)b * out_ld + cc;
   if (VEC) {
@@ -142,26 +121,30 @@ template <typename T, typename TO>
 void spmm_forward(const Launch& L, const int32_t* row_ptr, const int32_t* col, const float* val,
                   int64_t row0, int64_t group_row_stride, int G, int B, int64_t N0, const T* P,
                   int64_t p_ld, int64_t p_sg, const float* bias, int64_t bias_sg, int n1, TO* out,
-                  int64_t out_ld, int64_t out_sg, DeviceStatus* st) {
+                  int64_t out_ld, int64_t out_sg, DeviceStatus* st, bool relu) {
   dim3 grid((unsigned)ceil_div(B, kRowsPerCta), G, (unsigned)ceil_div(out_ld, 128));
   if (p_ld % 4 == 0 && out_ld % 4 == 0)
     spmm_forward_kernel<T, TO, true><<<grid, dim3(32, kRowsPerCta), 0, L.stream>>>(
         row_ptr, col, val, row0, group_row_stride, B, N0, P, p_ld, p_sg, bias, bias_sg, n1, out,
-        out_ld, out_sg, st);
+        out_ld, out_sg, st, relu);
   else
     spmm_forward_kernel<T, TO, false><<<grid, dim3(32, kRowsPerCta), 0, L.stream>>>(
         row_ptr, col, val, row0, group_row_stride, B, N0, P, p_ld, p_sg, bias, bias_sg, n1, out,
-        out_ld, out_sg, st);
+        out_ld, out_sg, st, relu);
   L.count();
 }
 template void spmm_forward<float, float>(const Launch&, const int32_t*, const int32_t*, const float*,
                                          int64_t, int64_t, int, int, int64_t, const float*, int64_t,
                                          int64_t, const float*, int64_t, int, float*, int64_t, int64_t,
-                                         DeviceStatus*);
+                                         DeviceStatus*, bool);
+template void spmm_forward<bf16, float>(const Launch&, const int32_t*, const int32_t*, const float*,
+                                        int64_t, int64_t, int, int, int64_t, const bf16*, int64_t,
+                                        int64_t, const float*, int64_t, int, float*, int64_t, int64_t,
+                                        DeviceStatus*, bool);
 template void spmm_forward<bf16, bf16>(const Launch&, const int32_t*, const int32_t*, const float*,
                                        int64_t, int64_t, int, int, int64_t, const bf16*, int64_t,
                                        int64_t, const float*, int64_t, int, bf16*, int64_t, int64_t,
-                                       DeviceStatus*);
+                                       DeviceStatus*, bool);
 
 template <typename T>
 void spmm_backward_sgd(const Launch& L, const int32_t* row_ptr, const int32_t* col, const float* val,

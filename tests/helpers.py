@@ -32,9 +32,9 @@ def make_problem(w: synth.Workload, bias_scale=0.1, round_index=0):
     return W, b, data
 
 
-def oracle_round(w: synth.Workload, W, b, data, seed, dtype=np.float64):
+def oracle_round(w: synth.Workload, W, b, data, seed, dtype=np.float64, norm_eps=None):
     from oracle import ist_oracle as O
-    o = O.IstOracle(w.layer_dims, w.S, dtype=dtype)
+    o = O.IstOracle(w.layer_dims, w.S, dtype=dtype, norm_eps=norm_eps)
     o.bind_weights(W, b)
     X = (data.row_ptr, data.col, data.val) if data.is_csr else data.X
     parts = o.partition(seed)
@@ -70,8 +70,10 @@ def gpu_inputs(w: synth.Workload, data, device="cuda:0", as_bf16=None):
     return X, y
 
 
-def gpu_round(w: synth.Workload, W, b, data, seed, device="cuda:0", as_bf16=None):
+def gpu_round(w: synth.Workload, W, b, data, seed, device="cuda:0", as_bf16=None, norm_eps=None):
     ctx, Wd, bd = gpu_context(w, W, b, device)
+    if norm_eps is not None:
+        ctx.enable_normalization(norm_eps)
     X, y = gpu_inputs(w, data, device, as_bf16)
     ctx.partition(seed)
     parts = [tuple(t.cpu().numpy() for t in ctx.get_partition(l)) for l in range(1, ctx.t)]

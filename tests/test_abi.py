@@ -59,3 +59,9 @@ def test_create_rejects_bad_workspace_without_a_device(api):
     st = api.lib.ist_create(ctypes.byref(h), dims, 3, 2, api.IST_FP32, 4, 0, ctypes.c_void_p(256), 16, None)
     assert st == api.IST_ERR_WORKSPACE
     assert api.lib.ist_partition(None, 1) == api.IST_ERR_ARG
+
+
+def test_normalisation_entry_points_reject_null_contexts(api):
+    assert api.lib.ist_norm_workspace_bytes(None) == 0
+    assert api.lib.ist_enable_normalization(None, ctypes.c_float(1e-5), None, 0) == api.IST_ERR_ARG
+    assert api.lib.ist_calibrate(None, None, 1) == api.IST_ERR_ARG
