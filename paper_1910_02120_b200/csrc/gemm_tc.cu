@@ -15,7 +15,9 @@
 //                      the epilogue, write the chunk into a swizzled shared-memory slot
 //   warp 10 (one lane) TMA loads of the epilogue's input chunks into the slots: the fp32 master
 //                      slice for the SGD update, the ReLU mask for the delta GEMM
-//   warp 11 (one lane) TMA stores of finished slots (coalesced, clipped at the tensor edge)
+//   warps 11..14 (one lane each) TMA stores of finished slots (coalesced, clipped at the tensor
+//                      edge); slot i belongs to storer i % 4, which hands the slot back as soon
+//                      as its own store has read it, without waiting for a later chunk
 // The epilogue has no CTA-wide barrier: slots move between loader, epilogue warps and storer
 // through mbarriers (slot_full -> chunk_done -> slot_empty), so warps work on different chunks
 // at the same time and a slow chunk does not hold the others back.
@@ -50,9 +52,10 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;                   // 64 bf16 = 128 bytes = one swizzle row
 constexpr int CH = 32;                   // epilogue chunk: 32 output columns
-constexpr int kThreads = 384;            // 12 warps, see the role list above
+constexpr int kThreads = 480;            // 15 warps, see the role list above
 constexpr int kEpiWarps = 8;
 constexpr int kAuxWarp = 10;
+constexpr int kStoreWarp0 = 11, kStoreWarps = 4;
 constexpr long long kWaitLimitCycles = 2000000000ll;   // ~1 s at 2 GHz
 
 // ---- small PTX wrappers ------------------------------------------------------------------------
@@ -556,6 +559,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else {
     // ---------------------------------------------------------------- chunk stores
     if (lane == 0) {
+      const int sj = warp - kStoreWarp0;
       int cq = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
@@ -566,16 +570,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const int nc = n0 + c * CH;
           if (nc >= a.N) break;
           const int slot = cq % NS;
+          // a slot always belongs to the same storer, so that storer sees the slot's barrier
+          // phases in order (a parity wait cannot tell phase p from phase p + 2)
+          if (slot % kStoreWarps != sj) continue;
           ok = mbar_wait(&chunk_done[slot], (cq / NS) & 1, abortp, a.status, 7);
           if (!ok) break;
           uint8_t* f32 = slots + slot * SLOT_BYTES;
           if (ET::k32) tma_store_3d(&tmC32, f32, nc, m0, g);
           if (ET::k16) tma_store_3d(&tmC16, f32 + F32_BYTES, nc, m0, g);
           tma_commit_group();
-          // one store may stay in flight; the slot of the one before it has been read and can be
-          // refilled (by the loader) or rewritten (by the epilogue warps)
-          tma_wait_read<1>();
-          if (cq >= 1) mbar_arrive(&slot_empty[(cq - 1) % NS]);
+          // once the store has read the slot it can be refilled (by the loader) or rewritten (by
+          // the epilogue warps); the write to global memory completes in the background
+          tma_wait_read<0>();
+          mbar_arrive(&slot_empty[slot]);
         }
       }
       tma_wait_all();                // all stores complete before the CTA exits
