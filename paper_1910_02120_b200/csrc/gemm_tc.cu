@@ -444,6 +444,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
       const int g = tile / (a.m_tiles * a.n_tiles);   // output slab (group, k slice)
       const int b = j & 1;
+      // Bias of the tile's columns, fetched while the tile's MMAs are still running (a load inside
+      // the chunk loop would cost an L2 round trip per chunk): lane l keeps column 32 * c + l of
+      // every chunk c, and the chunk code reads the 32 values of its chunk with warp shuffles.
+      float bias_reg[NCH];
+      if (EPI == EPI_BIAS_RELU || EPI == EPI_BIAS_F32) {
+        const float* bias = a.bias ? a.bias + (long long)(g / a.k_splits) * a.bias_sg : nullptr;
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const int n = n0 + c * CH + lane;
+          bias_reg[c] = (bias && n < a.N) ? __ldg(bias + n) : 0.f;
+        }
+      }
       // warp-uniform outcome: the tensor-memory loads below need the whole warp
       ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[b], (j >> 1) & 1, abortp, a.status, 4));
       if (!ok) break;
@@ -493,21 +505,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             *pm = pack8(o);
           }
         } else {
-          // bias of the tile's group; a k slice of a split product carries none
-          const float* bias = a.bias ? a.bias + (long long)(g / a.k_splits) * a.bias_sg : nullptr;
+          float bl = 0.f;   // this lane's bias value of chunk c (zero for a k slice of a split product)
+#pragma unroll
+          for (int i = 0; i < NCH; ++i)
+            if (i == c) bl = bias_reg[i];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
             float o[8];
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-              const int n = nc + 8 * u + 4 * hh;
-              float4 bv = (bias && n < a.N) ? __ldg(reinterpret_cast<const float4*>(bias + n))
-                                            : make_float4(0.f, 0.f, 0.f, 0.f);
-              o[4 * hh + 0] = __uint_as_float(acc[8 * u + 4 * hh + 0]) + bv.x;
-              o[4 * hh + 1] = __uint_as_float(acc[8 * u + 4 * hh + 1]) + bv.y;
-              o[4 * hh + 2] = __uint_as_float(acc[8 * u + 4 * hh + 2]) + bv.z;
-              o[4 * hh + 3] = __uint_as_float(acc[8 * u + 4 * hh + 3]) + bv.w;
-            }
+            for (int e = 0; e < 8; ++e)
+              o[e] = __uint_as_float(acc[8 * u + e]) + __shfl_sync(0xffffffffu, bl, 8 * u + e);
             if (EPI == EPI_BIAS_RELU) {
 #pragma unroll
               for (int e = 0; e < 8; ++e) o[e] = fmaxf(o[e], 0.f);
