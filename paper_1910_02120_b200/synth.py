@@ -102,6 +102,30 @@ def make_labels(shape, n_classes: int, seed: int) -> np.ndarray:
     return rng_for(seed, 7).integers(0, n_classes, size=shape, dtype=np.int32)
 
 
+def make_teacher_task(n_rows: int, N0: int, n_classes: int, seed: int, hidden: int = 32):
+    """A learnable classification task: X ~ N(0, 1) [n_rows][N0] fp32 and labels drawn by a fixed
+    random scoring function, y = argmax(tanh(X A / sqrt(N0)) C) with A [N0][hidden], C
+    [hidden][n_classes] ~ N(0, 1).  Stands in for a real dataset in multi-round runs (labels
+    that depend on the inputs, unlike make_labels)."""
+    g = rng_for(seed, 11)
+    X = g.standard_normal((n_rows, N0), dtype=np.float32)
+    A = g.standard_normal((N0, hidden))
+    C = g.standard_normal((hidden, n_classes))
+    scores = np.tanh(X.astype(np.float64) @ A / np.sqrt(N0)) @ C
+    return X, scores.argmax(axis=1).astype(np.int32)
+
+
+def draw_round_rows(n_rows: int, S: int, K: int, B: int, seed: int, round_index: int) -> np.ndarray:
+    """Row indices [S][K][B] of the minibatches of one round: uniform draws without replacement
+    inside a batch, independent across subnets, steps and rounds."""
+    g = rng_for(seed, 1000 + round_index)
+    out = np.empty((S, K, B), dtype=np.int64)
+    for s in range(S):
+        for k in range(K):
+            out[s, k] = g.choice(n_rows, size=B, replace=False)
+    return out
+
+
 def make_dense_inputs(S: int, K: int, B: int, N0: int, dist: str, seed: int) -> np.ndarray:
     """X laid out as [S][K][B][N0] fp32: one distinct batch per subnet per step."""
     g = rng_for(seed, 3)
