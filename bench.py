@@ -44,6 +44,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C3", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--shard-subnets", action="store_true",
+                    help="with --gpus N > 1: split the S subnets over the ranks (one all-gather of the trained "
+                         "slices per round, strong scaling) instead of running N independent replicas")
     ap.add_argument("--norm-eps", type=float, default=None,
                     help="standardise hidden pre-activations over the batch (Sec. 2.2) with this epsilon")
     ap.add_argument("--local-steps", type=int, default=0,
@@ -69,7 +72,7 @@ def peaks():
     return p
 
 
-def config_dict(w: synth.Workload, n_gpus: int, norm_eps=None):
+def config_dict(w: synth.Workload, n_gpus: int, norm_eps=None, sharded=False):
     extra = {} if norm_eps is None else {"normalization": f"per-neuron batch standardisation, eps={norm_eps:g}"}
     return {
         **extra,
@@ -79,7 +82,9 @@ def config_dict(w: synth.Workload, n_gpus: int, norm_eps=None):
         "step": "one IST round: partition+gather, K local SGD steps of S subnets, reassemble",
         "inputs": f"{w.x_dist}; distinct batch per subnet per local step",
         "l2": "per-round working set (inputs + full network + packed slices) exceeds the 126 MB L2",
-        "parallelism": "single GPU" if n_gpus == 1 else f"{n_gpus} independent replicas",
+        "parallelism": "single GPU" if n_gpus == 1 else
+                       (f"{w.S} subnets split over {n_gpus} GPUs, one all-gather of trained slices per round" if sharded
+                        else f"{n_gpus} independent replicas"),
     }
 
 
@@ -283,17 +288,28 @@ def run_ours(args, w):
         dist.init_process_group("nccl", device_id=dev)
 
     # ---- inputs, resident on the device before timing starts ---------------------------------
-    ww = w.scaled(seed=w.seed + 1000 * rank)
+    shard = args.shard_subnets and world > 1
+    if shard:
+        from paper_1910_02120_b200 import sharding
+        first, count = sharding.subnet_range(w.S, world, rank)
+    ww = w.scaled(seed=w.seed + (0 if shard else 1000 * rank))
     W, b = synth.make_weights(ww.layer_dims, ww.seed)
     Wd = [torch.from_numpy(x).to(dev) for x in W]
     bd = [torch.from_numpy(x).to(dev) for x in b]
     del W, b
     data = synth.make_round_inputs(ww)
+    if shard:      # same network and partition everywhere; this rank keeps the rows of its own subnets
+        if data.is_csr:
+            raise SystemExit("--shard-subnets takes dense inputs")
+        data = synth.Batchset(y=data.y[first:first + count].copy(), X=data.X[first:first + count].copy())
     prec = api.IST_BF16 if w.precision == "bf16" else api.IST_FP32
     ctx = api.Ist(w.layer_dims, w.S, prec, w.B, input_is_csr=data.is_csr, device=str(dev))
     ctx.bind_weights(Wd, bd)
     if args.norm_eps is not None:
         ctx.enable_normalization(args.norm_eps)
+    if shard:
+        ctx.set_subnet_range(first, count)
+    n_local = count if shard else w.S
     y_host = torch.from_numpy(data.y.reshape(-1).copy()).pin_memory()
     if data.is_csr:
         host_in = [torch.from_numpy(data.row_ptr.astype(np.int32)).pin_memory(),
@@ -305,8 +321,8 @@ def run_ours(args, w):
         host_in = [xt.pin_memory()]
     dev_in = [t.to(dev) for t in host_in]
     y_dev = y_host.to(dev)
-    loss_dev = torch.empty(w.S * w.K, dtype=torch.float32, device=dev)
-    loss_host = torch.empty(w.S * w.K, dtype=torch.float32).pin_memory()
+    loss_dev = torch.empty(n_local * w.K, dtype=torch.float32, device=dev)
+    loss_host = torch.empty(n_local * w.K, dtype=torch.float32).pin_memory()
     h2d = sum(t.numel() * t.element_size() for t in host_in) + y_host.numel() * 4
     d2h = loss_host.numel() * 4
 
@@ -314,7 +330,10 @@ def run_ours(args, w):
         return tuple(ts) if data.is_csr else ts[0]
 
     def one_round(r, X, y):
-        ctx.round(7000 + r, X, y, w.lr, w.K, w.B, loss_out=loss_dev)
+        if shard:
+            sharding.sharded_round(ctx, 7000 + r, X, y, w.lr, w.K, w.B, first, count, loss_out=loss_dev)
+        else:
+            ctx.round(7000 + r, X, y, w.lr, w.K, w.B, loss_out=loss_dev)
 
     def barrier():
         if world > 1:
@@ -340,12 +359,13 @@ def run_ours(args, w):
     clocks = sampler.stop()
     ms = max_over_ranks(e0.elapsed_time(e1), dev)
     ctx.sync_status()
-    value = job_value(w.samples_per_round, args.steps, world, ms)
+    per_rank = w.samples_per_round // world if shard else w.samples_per_round   # samples this rank's subnets saw
+    value = job_value(per_rank, args.steps, world, ms)
     if args.quick:
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                               "warmup": n_warm, "ms_per_step": ms / args.steps, "quick": True,
-                              "gpu_launches": launches, "config": config_dict(w, world, args.norm_eps)}))
+                              "gpu_launches": launches, "config": config_dict(w, world, args.norm_eps, shard)}))
         if world > 1:
             dist.destroy_process_group()
         return
@@ -383,7 +403,7 @@ def run_ours(args, w):
     e1.record()
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1), dev)
-    e2e_value = job_value(w.samples_per_round, args.steps, world, ms_e2e)
+    e2e_value = job_value(per_rank, args.steps, world, ms_e2e)
 
     # ---- per-kernel-class device times (separate pass, events around each class) ---------------
     ctx.profile(True)
@@ -401,6 +421,12 @@ def run_ours(args, w):
 
     pk = peaks()
     wm = work_model(w, norm=args.norm_eps is not None)
+    if shard:      # this rank ran the local steps of its own subnets only; gather / scatter cover all S
+        for k in ("fwd", "dx", "dw_sgd"):
+            wm["flops"][k] = wm["flops"][k] * count // w.S
+        for k in ("dw_sgd", "norm"):
+            if k in wm["bytes"]:
+                wm["bytes"][k] = wm["bytes"][k] * count // w.S
     tensor_peak = pk["bf16_tflops_sustained"] if w.precision == "bf16" else None
     kernels = {}
     for name, (n, t_ms) in prof.items():
@@ -461,8 +487,9 @@ def run_ours(args, w):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": n_warm, "ms_per_step": ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": w.precision.replace("fp", "f"), "data": "synthetic",
-        "config": config_dict(w, world, args.norm_eps), "clocks": clocks,
+        "scaling": "strong" if shard else "weak", "vs_baseline": None, "dtype": w.precision.replace("fp", "f"),
+        "data": "synthetic",
+        "config": config_dict(w, world, args.norm_eps, shard), "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": launches, "roofline": roof, "kernels": kernels, "cpu_baseline": cpu,

@@ -142,6 +142,25 @@ ist_status ist_local_steps(ist_ctx* ctx, const ist_input* X, const int32_t* y_de
                            float* loss_out_dev);
 
 /*
+ * Training the S subnets at several sites (Sec. 2.1: "Each of the n subnets is sent to a compute
+ * node"; Sec. 2.3: only the slices travel).  A context may train only subnets first .. first +
+ * count - 1 in ist_local_steps; the other subnets' slices are trained by other contexts (other
+ * GPUs, one process each) that hold a copy of the same full network and draw the same
+ * partition (same seed).  Before ist_reassemble every context must hold all S trained slices:
+ * ist_packed_layer gives the device address of layer l's packed fp32 slices
+ * ([S][*master_bytes_per_subnet], subnet s at byte offset s * bytes) and of its packed biases,
+ * so that the caller can exchange them (one all-gather per layer over the subnet dimension, each
+ * site contributing its own `count` slabs).  ist_partition still gathers all S slices and
+ * ist_reassemble still writes all S back; only ist_local_steps is narrowed.
+ * In ist_local_steps the inputs and losses are then addressed by the local subnet index
+ * (0 .. count-1): rows start at i * stride_subnet, loss_out_dev holds count * K values.
+ * Default range: all S subnets.  Not allowed while a partition is in place.
+ */
+ist_status ist_set_subnet_range(ist_ctx* ctx, int first, int count);
+ist_status ist_packed_layer(ist_ctx* ctx, int layer, void** master_dev, size_t* master_bytes_per_subnet,
+                            void** bias_dev, size_t* bias_bytes_per_subnet);
+
+/*
  * Sec. 2.1: "subnet parameters are copied back into the full NN, where no collisions occur".
  * Writes every trained slice to the positions it was gathered from; entries of middle layers
  * whose row group differs from their column group are not written.  The output bias, the one

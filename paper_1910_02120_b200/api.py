@@ -25,6 +25,7 @@ EXPORTS = [
     "ist_get_subnet_params", "ist_local_steps", "ist_reassemble", "ist_eval", "ist_sync_status",
     "ist_kernel_launches", "ist_last_error", "ist_destroy", "ist_profile", "ist_profile_read",
     "ist_partition_layer_static", "ist_norm_workspace_bytes", "ist_enable_normalization", "ist_calibrate",
+    "ist_set_subnet_range", "ist_packed_layer",
 ]
 IST_STATIC_MAX_NEURONS, IST_STATIC_MAX_SUBNETS = 65536, 64
 
@@ -96,6 +97,11 @@ def _load() -> ctypes.CDLL:
     lib.ist_enable_normalization.restype = i32
     lib.ist_calibrate.argtypes = [vp, ctypes.POINTER(IstInput), i64]
     lib.ist_calibrate.restype = i32
+    lib.ist_set_subnet_range.argtypes = [vp, i32, i32]
+    lib.ist_set_subnet_range.restype = i32
+    lib.ist_packed_layer.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(sz), ctypes.POINTER(vp),
+                                     ctypes.POINTER(sz)]
+    lib.ist_packed_layer.restype = i32
     lib.ist_destroy.argtypes = [vp]
     return lib
 
@@ -249,11 +255,12 @@ class Ist:
             stride_step = batch
         inp, keep = make_input(X, batch, stride_subnet, stride_step)
         assert y.is_cuda and y.dtype == torch.int32 and y.is_contiguous()
+        n_sub = getattr(self, "sub_count", self.S)
         if loss_out is None and want_loss:
-            loss_out = torch.empty(self.S * K, dtype=torch.float32, device=self.device)
+            loss_out = torch.empty(n_sub * K, dtype=torch.float32, device=self.device)
         _check(self.handle, lib.ist_local_steps(self.handle, ctypes.byref(inp), y.data_ptr(),
                                                 ctypes.c_float(lr), K, _ptr(loss_out)))
-        return loss_out.view(self.S, K) if loss_out is not None else None
+        return loss_out.view(n_sub, K) if loss_out is not None else None
 
     def reassemble(self):
         _check(self.handle, lib.ist_reassemble(self.handle))
@@ -265,6 +272,24 @@ class Ist:
         _check(self.handle, lib.ist_eval(self.handle, ctypes.byref(inp), y.data_ptr(), n,
                                          loss.data_ptr(), correct.data_ptr()))
         return loss, correct
+
+    def set_subnet_range(self, first: int, count: int):
+        """Train only subnets first .. first+count-1 in local_steps (the others are trained elsewhere)."""
+        _check(self.handle, lib.ist_set_subnet_range(self.handle, first, count))
+        self.sub_first, self.sub_count = first, count
+
+    def packed_layer(self, layer: int):
+        """(master [S][elems] fp32, bias [S][ld] fp32): views of the workspace, for the slice exchange."""
+        mp, mb, bp, bb = ctypes.c_void_p(), ctypes.c_size_t(), ctypes.c_void_p(), ctypes.c_size_t()
+        _check(self.handle, lib.ist_packed_layer(self.handle, layer, ctypes.byref(mp), ctypes.byref(mb),
+                                                 ctypes.byref(bp), ctypes.byref(bb)))
+        base = self.workspace.data_ptr()
+
+        def view(ptr, nbytes):
+            off = ptr.value - base
+            return self.workspace[off:off + self.S * nbytes].view(torch.float32).view(self.S, nbytes // 4)
+
+        return view(mp, mb.value), view(bp, bb.value)
 
     def enable_normalization(self, eps: float):
         """Sec. 2.2 batch standardisation of the hidden layers for all later calls."""

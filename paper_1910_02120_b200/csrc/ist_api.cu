@@ -67,6 +67,9 @@ struct ist_ctx {
   uint64_t seed = 0;
   std::string err;
 
+  // subnets this context trains in ist_local_steps (all S unless ist_set_subnet_range narrowed it)
+  int sub_first = 0, sub_count = 0;
+
   // batch standardisation of hidden pre-activations (off unless ist_enable_normalization ran)
   bool norm = false, calibrated = false;
   float norm_eps = 0.f;
@@ -227,6 +230,8 @@ void make_norm_plan(ist_ctx* c) {
 void fill_shape(ist_ctx* c, const int64_t* dims, int n_dims, int S, int precision, int max_batch, int csr) {
   c->t = n_dims - 1;
   c->S = S;
+  c->sub_first = 0;
+  c->sub_count = S;
   c->precision = precision;
   c->max_batch = max_batch;
   c->csr = csr ? 1 : 0;
@@ -349,13 +354,18 @@ void small_softmax(const Launch& L, const float* part, int ks, int64_t ld, int G
 template <typename T>
 ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, float lr, int K,
                            float* loss_out) {
-  const int t = c->t, S = c->S, B = X->batch;
+  // S here is the number of subnets this context trains: slabs s0 .. s0 + S - 1 of the packed
+  // weights; activations, deltas and the other scratch buffers use their first S slabs.
+  const int t = c->t, S = c->sub_count, s0 = c->sub_first, B = X->batch;
   const int64_t Bm = c->max_batch;
   const bool bf = c->precision == IST_BF16;
   auto act = [&](int l) { return c->plan.act[l].at<T>(c->ws); };
   auto delta = [&](int l) { return c->plan.delta[l].at<T>(c->ws); };
+  auto master = [&](int l) { return c->master(l) + (int64_t)s0 * c->slice_elems(l); };
+  auto opw = [&](int l) -> bf16* { return bf ? c->opw(l) + (int64_t)s0 * c->slice_elems(l) : nullptr; };
+  auto bias_of = [&](int l) { return c->bias(l) + (int64_t)s0 * c->ld[l]; };
   auto weights = [&](int l) -> const T* {       // operand copy of layer l's slices
-    return bf ? reinterpret_cast<const T*>(c->opw(l)) : reinterpret_cast<const T*>(c->master(l));
+    return bf ? reinterpret_cast<const T*>(opw(l)) : reinterpret_cast<const T*>(master(l));
   };
   float* logits = c->plan.logits.at<float>(c->ws);
   float* row_loss = c->plan.row_loss.at<float>(c->ws);
@@ -401,11 +411,11 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
           Scope sc(c, IST_K_SPMM);
           if (c->norm)
             spmm_forward<T, float>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
-                                   weights(1), c->ld[1], c->slice_elems(1), c->bias(1), c->ld[1],
+                                   weights(1), c->ld[1], c->slice_elems(1), bias_of(1), c->ld[1],
                                    (int)c->np[1], c->zbuf(1), c->ld[1], Bm * c->ld[1], st, false);
           else
             spmm_forward<T, T>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
-                               weights(1), c->ld[1], c->slice_elems(1), c->bias(1), c->ld[1],
+                               weights(1), c->ld[1], c->slice_elems(1), bias_of(1), c->ld[1],
                                (int)c->np[1], act(1), c->ld[1], Bm * c->ld[1], st);
         }
         if (c->norm) standardise(1);
@@ -416,7 +426,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       g.N_store = (int)c->ld[l];
       g.A = in_ptr(l - 1); g.a_sm = in_ld(l - 1); g.a_sk = 1; g.a_sg = in_sg(l - 1);
       g.B = weights(l); g.b_sn = 1; g.b_sk = c->ld[l]; g.b_sg = c->slice_elems(l);
-      g.bias = c->bias(l); g.bias_sg = c->ld[l];
+      g.bias = bias_of(l); g.bias_sg = c->ld[l];
       if (l < t && c->norm) {
         g.epi = EPI_BIAS_F32;        // fp32 pre-activations; standardisation and ReLU follow
         g.outf = c->zbuf(l); g.outf_ld = c->ld[l]; g.outf_sg = Bm * c->ld[l];
@@ -442,7 +452,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
     {
       Scope sc(c, IST_K_LOSS);
       if (head)
-        small_softmax(L, logits, head_ks, c->ld[t], S, B, (int)c->N[t], c->bias(t), c->ld[t], y + row0,
+        small_softmax(L, logits, head_ks, c->ld[t], S, B, (int)c->N[t], bias_of(t), c->ld[t], y + row0,
                       X->stride_subnet, delta(t), c->ld[t], Bm * c->ld[t], row_loss, st);
       else
       softmax_xent<T>(L, logits, c->ld[t], Bm * c->ld[t], S, B, (int)c->N[t], y + row0,
@@ -455,7 +465,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       BiasSgdArgs<T> ba{};
       int n = 0;
       for (int l = l_hi; l >= l_lo; --l) {
-        ba.layer[n++] = BiasSgdLayer<T>{delta(l), c->ld[l], Bm * c->ld[l], c->bias(l), c->ld[l], (int)c->np[l]};
+        ba.layer[n++] = BiasSgdLayer<T>{delta(l), c->ld[l], Bm * c->ld[l], bias_of(l), c->ld[l], (int)c->np[l]};
         if (n == kMaxBiasLayers || l == l_lo) {
           bias_sgd<T>(L, ba, n, S, B, lr);
           n = 0;
@@ -489,7 +499,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {
         Scope sc(c, IST_K_SPMM);
         spmm_backward_sgd<T>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
-                             delta(1), c->ld[1], Bm * c->ld[1], (int)c->np[1], c->master(1), c->opw(1),
+                             delta(1), c->ld[1], Bm * c->ld[1], (int)c->np[1], master(1), opw(1),
                              c->ld[1], c->slice_elems(1), lr);
         continue;
       }
@@ -499,8 +509,8 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       g.A = in_ptr(l - 1); g.a_sm = 1; g.a_sk = in_ld(l - 1); g.a_sg = in_sg(l - 1);
       g.B = delta(l); g.b_sn = 1; g.b_sk = c->ld[l]; g.b_sg = Bm * c->ld[l];
       g.epi = EPI_SGD;
-      g.outf = c->master(l); g.outf_ld = c->ld[l]; g.outf_sg = c->slice_elems(l);
-      g.opw = c->opw(l);
+      g.outf = master(l); g.outf_ld = c->ld[l]; g.outf_sg = c->slice_elems(l);
+      g.opw = opw(l);
       g.lr = lr;
       Scope sc(c, IST_K_DW_SGD);
       if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "weight-gradient GEMM of layer %d cannot be launched", l);
@@ -642,6 +652,28 @@ extern "C" ist_status ist_local_steps(ist_ctx* c, const ist_input* X, const int3
   if (s != IST_OK) return s;
   if (c->precision == IST_BF16) return run_local_steps<bf16>(c, X, y_dev, lr, K, loss_out_dev);
   return run_local_steps<float>(c, X, y_dev, lr, K, loss_out_dev);
+}
+
+extern "C" ist_status ist_set_subnet_range(ist_ctx* c, int first, int count) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state == ST_PARTITIONED)
+    return fail(c, IST_ERR_STATE, "the subnet range cannot change between ist_partition and ist_reassemble");
+  if (first < 0 || count < 1 || first > c->S - count)
+    return fail(c, IST_ERR_ARG, "subnet range [%d, %d) outside [0, %d)", first, first + count, c->S);
+  c->sub_first = first;
+  c->sub_count = count;
+  return IST_OK;
+}
+
+extern "C" ist_status ist_packed_layer(ist_ctx* c, int layer, void** master_dev, size_t* master_bytes_per_subnet,
+                                       void** bias_dev, size_t* bias_bytes_per_subnet) {
+  if (!c) return IST_ERR_ARG;
+  if (layer < 1 || layer > c->t) return fail(c, IST_ERR_ARG, "layer outside 1..t");
+  if (master_dev) *master_dev = c->master(layer);
+  if (master_bytes_per_subnet) *master_bytes_per_subnet = (size_t)c->slice_elems(layer) * 4;
+  if (bias_dev) *bias_dev = c->bias(layer);
+  if (bias_bytes_per_subnet) *bias_bytes_per_subnet = (size_t)c->ld[layer] * 4;
+  return IST_OK;
 }
 
 extern "C" ist_status ist_reassemble(ist_ctx* c) {

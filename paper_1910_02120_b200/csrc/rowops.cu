@@ -219,6 +219,7 @@ __global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int B, 
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (c0 < L.ld) {
     const T* d = L.delta + (int64_t)g * L.sg + c0;
+#pragma unroll 8
     for (int b = ry; b < B; b += 32) {
       float v[8];
       load8(d + (int64_t)b * L.ld, v);
