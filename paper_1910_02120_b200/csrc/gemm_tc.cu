@@ -220,6 +220,12 @@ struct TcArgs {
   const float* bias; long long bias_sg;
   float lr;
   DeviceStatus* status;
+  // wide softmax head (see GemmArgs)
+  float2* lse_part;
+  const float* lse; long long lse_sg;
+  const int32_t* labels; long long labels_sg;
+  float* label_logit;
+  float inv_rows;
 };
 
 // Chunk staging: a ring of fp32 areas ([128][32] floats, 128-byte swizzle) and / or a ring of
@@ -230,7 +236,14 @@ template <> struct EpiTraits<EPI_BIAS_RELU> { static constexpr bool k32 = false,
 template <> struct EpiTraits<EPI_BIAS_F32> { static constexpr bool k32 = true, k16 = false, kAux = false; };
 template <> struct EpiTraits<EPI_RELU_MASK> { static constexpr bool k32 = false, k16 = true, kAux = true; };
 template <> struct EpiTraits<EPI_SGD> { static constexpr bool k32 = true, k16 = true, kAux = true; };
+template <> struct EpiTraits<EPI_LSE_PART> { static constexpr bool k32 = false, k16 = false, kAux = false; };
+template <> struct EpiTraits<EPI_SOFTMAX_DELTA> { static constexpr bool k32 = false, k16 = true, kAux = false; };
 
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint4 pack8(const float* v) {
   __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
   __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
@@ -273,6 +286,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   constexpr uint32_t AUX_BYTES = EPI == EPI_SGD ? F32_BYTES : B16_BYTES;
   constexpr uint32_t TMEM_COLS = 2 * BN;
   constexpr int NCH = BN / CH;
+  constexpr bool kStore = ET::k32 || ET::k16;   // the epilogue writes chunks through the slot ring
+  constexpr float kLog2e = 1.4426950408889634f;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -440,22 +455,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int r = q * 32 + lane;                      // row of the tile owned by this thread
     int cq = 0, j = 0;
     bool ok = true;
-    for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
+    // per-tile epilogue inputs, requested one tile ahead (see below)
+    float next_bias[NCH];
+    float next_lse = 0.f;
+    int next_label = -1;
+    auto prefetch_tile_inputs = [&](int tile) {
       const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
-      const int g = tile / (a.m_tiles * a.n_tiles);   // output slab (group, k slice)
-      const int b = j & 1;
-      // Bias of the tile's columns, fetched while the tile's MMAs are still running (a load inside
-      // the chunk loop would cost an L2 round trip per chunk): lane l keeps column 32 * c + l of
-      // every chunk c, and the chunk code reads the 32 values of its chunk with warp shuffles.
-      float bias_reg[NCH];
-      if (EPI == EPI_BIAS_RELU || EPI == EPI_BIAS_F32) {
+      const int g = tile / (a.m_tiles * a.n_tiles);
+      if (EPI == EPI_BIAS_RELU || EPI == EPI_BIAS_F32 || EPI == EPI_LSE_PART || EPI == EPI_SOFTMAX_DELTA) {
         const float* bias = a.bias ? a.bias + (long long)(g / a.k_splits) * a.bias_sg : nullptr;
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           const int n = n0 + c * CH + lane;
-          bias_reg[c] = (bias && n < a.N) ? __ldg(bias + n) : 0.f;
+          next_bias[c] = (bias && n < a.N) ? __ldg(bias + n) : 0.f;
         }
       }
+      if (EPI == EPI_SOFTMAX_DELTA) {
+        const int row = (tile % a.m_tiles) * (BM * PAIR) + rank * BM + r;
+        next_lse = row < a.M ? __ldg(a.lse + (long long)g * a.lse_sg + row) : 0.f;
+        next_label = row < a.M ? __ldg(a.labels + (long long)g * a.labels_sg + row) : -1;
+      }
+    };
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) next_bias[c] = 0.f;
+    if (unit < total_tiles) prefetch_tile_inputs(unit);
+    for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
+      const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
+      const int g = tile / (a.m_tiles * a.n_tiles);   // output slab (group, k slice)
+      const int b = j & 1;
+      // Bias of the tile's columns: lane l keeps column 32 * c + l of every chunk c, and the chunk
+      // code reads the 32 values of its chunk with warp shuffles.  The values (and the per-row
+      // inputs of the softmax pass) were requested one tile ahead, so that their L2 round trip is
+      // not paid inside a tile; the requests for the next tile go out now.
+      float bias_reg[NCH];
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) bias_reg[c] = next_bias[c];
+      const int row = (tile % a.m_tiles) * (BM * PAIR) + rank * BM + r;   // this thread's row of the output
+      float run_max = -INFINITY, run_sum = 0.f;       // EPI_LSE_PART: over this warp group's chunks
+      const float row_lse = next_lse * kLog2e;        // log-sum-exp in the log2 domain
+      const int row_label = next_label;
+      if (tile + n_units < total_tiles) prefetch_tile_inputs(tile + n_units);
       // warp-uniform outcome: the tensor-memory loads below need the whole warp
       ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[b], (j >> 1) & 1, abortp, a.status, 4));
       if (!ok) break;
@@ -469,10 +508,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint8_t* f32 = slots + slot * SLOT_BYTES;
         uint8_t* b16 = f32 + F32_BYTES;
         // the slot is ready: loaded (input chunk) or drained by the store of an earlier chunk
-        if (ET::kAux) ok = mbar_wait(&slot_full[slot], (cq / NS) & 1, abortp, a.status, 5);
-        else ok = mbar_wait(&slot_empty[slot], ((cq / NS) & 1) ^ 1, abortp, a.status, 5);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        if (kStore) {
+          if (ET::kAux) ok = mbar_wait(&slot_full[slot], (cq / NS) & 1, abortp, a.status, 5);
+          else ok = mbar_wait(&slot_empty[slot], ((cq / NS) & 1) ^ 1, abortp, a.status, 5);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        }
         uint32_t acc[32];
         tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * CH), acc);
         if (EPI == EPI_SGD) {
@@ -504,6 +545,60 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int e = 0; e < 8; ++e) o[e] = mk[e] > 0.f ? __uint_as_float(acc[8 * u + e]) : 0.f;
             *pm = pack8(o);
           }
+        } else if (EPI == EPI_LSE_PART || EPI == EPI_SOFTMAX_DELTA) {
+          // Both passes work on z * log2(e), so that every exponential is one ex2 and the scaling
+          // rides on the multiply-add that also adds the bias.
+          float bl = 0.f;
+#pragma unroll
+          for (int i = 0; i < NCH; ++i)
+            if (i == c) bl = bias_reg[i];
+          bl *= kLog2e;
+          float z[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            z[e] = fmaf(__uint_as_float(acc[e]), kLog2e, __shfl_sync(0xffffffffu, bl, e));
+          if (EPI == EPI_LSE_PART) {
+            // running (max, sum of 2^(z - max)) of this row over the chunks this warp group sees
+            if (nc + CH > a.N) {                         // CTA-uniform: the last, ragged chunk
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (nc + e >= a.N) z[e] = -INFINITY;     // pad columns do not count
+            }
+            // four independent chains each, so that the maxima, the ex2 and the sums overlap
+            float m4[4] = {z[0], z[1], z[2], z[3]};
+#pragma unroll
+            for (int e = 4; e < 32; ++e) m4[e & 3] = fmaxf(m4[e & 3], z[e]);
+            const float mn = fmaxf(run_max, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));   // finite: column nc is inside N
+            float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int e = 0; e < 32; ++e) s4[e & 3] += ex2_approx(z[e] - mn);
+            run_sum = fmaf(run_sum, ex2_approx(run_max - mn), (s4[0] + s4[1]) + (s4[2] + s4[3]));
+            run_max = mn;
+          } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              float o[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) o[e] = ex2_approx(z[8 * u + e] - row_lse) * a.inv_rows;
+              *b16_unit(b16, r, u) = pack8(o);
+            }
+            if (nc + CH > a.N) {                         // zero the pad columns of the ragged chunk
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (nc + e >= a.N)
+                  reinterpret_cast<bf16*>(b16_unit(b16, r, e >> 3))[e & 7] = __float2bfloat16_rn(0.f);
+            }
+            const int at = row_label - nc;               // the label's column, if it is in this chunk
+            if (at >= 0 && at < CH && row < a.M) {
+              float zl = 0.f;
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (e == at) zl = z[e];
+              reinterpret_cast<bf16*>(b16_unit(b16, r, at >> 3))[at & 7] =
+                  __float2bfloat16_rn((ex2_approx(zl - row_lse) - 1.f) * a.inv_rows);
+              a.label_logit[(long long)g * a.lse_sg + row] = zl * 0.6931471805599453f;
+            }
+          }
         } else {
           float bl = 0.f;   // this lane's bias value of chunk c (zero for a k slice of a split product)
 #pragma unroll
@@ -525,11 +620,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
         }
-        fence_async_smem();          // generic-proxy writes -> visible to the TMA store
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&chunk_done[slot]);
+        if (kStore) {
+          fence_async_smem();          // generic-proxy writes -> visible to the TMA store
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&chunk_done[slot]);
+        }
       }
       if (!ok) break;
+      if (EPI == EPI_LSE_PART && row < a.M) {
+        // two partials per tile (one per warp group), combined by lse_combine
+        const int tn = (tile / a.m_tiles) % a.n_tiles;
+        a.lse_part[((long long)g * (2 * a.n_tiles) + 2 * tn + wg) * a.M + row] = make_float2(run_max, run_sum);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {   // the accumulator is free again: tell the CTA that issues the MMAs
@@ -565,7 +667,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else {
     // ---------------------------------------------------------------- chunk stores
-    if (lane == 0) {
+    if (kStore && lane == 0) {
       const int sj = warp - kStoreWarp0;
       int cq = 0;
       bool ok = true;
@@ -753,6 +855,9 @@ TileChoice pick_tile(int M, int N, int G, int epi) {
   return {64, 1};
 }
 
+// Partials per row the EPI_LSE_PART epilogue writes: two per 256-column tile.
+int gemm_tc_lse_parts(int64_t n_store) { return 2 * (int)ceil_div(n_store, 256); }
+
 // Number of k slices gemm_tc will really use when `want` are asked for (slices hold whole
 // 64-deep k blocks, so the count can come out smaller).
 int gemm_tc_splits(int K, int want) {
@@ -766,7 +871,9 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
   const bool a_mn = a.a_sm == 1 && a.a_sk != 1, b_mn = a.b_sn == 1 && a.b_sk != 1;
   if (!a_mn && a.a_sk != 1) return false;
   if (!b_mn && a.b_sk != 1) return false;
-  const TileChoice tc = pick_tile(a.M, n_store, a.G * (a.k_splits > 1 ? a.k_splits : 1), a.epi);
+  TileChoice tc = pick_tile(a.M, n_store, a.G * (a.k_splits > 1 ? a.k_splits : 1), a.epi);
+  if (a.epi == EPI_LSE_PART || a.epi == EPI_SOFTMAX_DELTA)   // the partials are laid out per 256-column tile
+    tc = TileChoice{256, a.M > BM ? 2 : 1};
   const int bn = tc.bn, pair = tc.pair;
   TcArgs t{};
   t.M = a.M; t.N = n_store; t.K = a.K;
@@ -786,6 +893,11 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
   t.bias = a.bias; t.bias_sg = a.bias_sg;
   t.lr = a.lr;
   t.status = st;
+  t.lse_part = reinterpret_cast<float2*>(a.lse_part);
+  t.lse = a.lse; t.lse_sg = a.lse_sg;
+  t.labels = a.labels; t.labels_sg = a.labels_sg;
+  t.label_logit = a.label_logit;
+  t.inv_rows = a.inv_rows;
   if ((long long)t.m_tiles * t.n_tiles * t.G > 0x7fffffffll) return false;
 
   Maps m{};
@@ -823,6 +935,15 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
       if (bn == 256) return launch<0, 1, 256, 4, 2, EPI_BIAS_F32, 1>(L, m, t);
       if (bn == 128) return launch<0, 1, 128, 5, 3, EPI_BIAS_F32, 1>(L, m, t);
       return launch<0, 1, 64, 6, 3, EPI_BIAS_F32, 1>(L, m, t);
+    case EPI_LSE_PART:
+      if (a_mn || !b_mn || a.k_splits > 1 || !a.lse_part) return false;
+      if (pair == 2) return launch<0, 1, 256, 4, 1, EPI_LSE_PART, 2>(L, m, t);
+      return launch<0, 1, 256, 3, 1, EPI_LSE_PART, 1>(L, m, t);
+    case EPI_SOFTMAX_DELTA:
+      if (a_mn || !b_mn || a.k_splits > 1 || !a.lse || !a.labels || !a.label_logit) return false;
+      if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
+      if (pair == 2) return launch<0, 1, 256, 4, 6, EPI_SOFTMAX_DELTA, 2>(L, m, t);
+      return launch<0, 1, 256, 3, 6, EPI_SOFTMAX_DELTA, 1>(L, m, t);
     case EPI_RELU_MASK:
       if (a_mn || b_mn) return false;
       if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;

@@ -26,7 +26,7 @@ struct Region {
 // Placement of everything that lives in the caller's workspace blob.
 struct Plan {
   size_t total = 0;
-  Region status, part, row_loss, logits, ev_a, ev_b, ev_acc, splitk;
+  Region status, part, row_loss, logits, ev_a, ev_b, ev_acc, splitk, lse, label_logit;
   std::vector<Region> idx, off;             // hidden layer l at [l]  (1..t-1)
   std::vector<Region> master, bias, opw;    // layer l at [l]         (1..t)
   std::vector<Region> act, delta;           // act [0..t-1], delta [1..t]
@@ -168,6 +168,10 @@ int head_splits(const ist_ctx* c) {
   return (int)std::max<int64_t>(1, std::min<int64_t>(kHeadSplitsMax, nkb / 4));
 }
 
+// A very wide output layer (bf16 operands): the logits are never stored.  The product is formed
+// twice, once for per-row log-sum-exp partials and once for delta = (softmax - onehot) / B.
+bool wide_head(const ist_ctx* c) { return c->precision == IST_BF16 && c->ld[c->t] > 8192; }
+
 // delta_{l-1} = delta_l * W_l^T contracts over the width of layer l.  When that width is huge
 // (hundreds of thousands of classes) and the output small, the product has too few tiles to
 // fill the machine, so the contraction is cut into slices that run as separate tiles.
@@ -199,8 +203,13 @@ void make_plan(ist_ctx* c) {
   if (!c->csr) p.act[0] = p.take((size_t)S * Bm * c->ld[0] * es);   // staging of fp32 inputs
   for (int l = 1; l < t; ++l) p.act[l] = p.take((size_t)S * Bm * c->ld[l] * es);
   for (int l = 1; l <= t; ++l) p.delta[l] = p.take((size_t)S * Bm * c->ld[l] * es);
-  p.logits = p.take((size_t)S * Bm * c->ld[t] * 4 * (narrow_head(c) ? kHeadSplitsMax : 1));
+  if (wide_head(c))   // (max, sum) partials per row and 128 columns instead of the logits themselves
+    p.logits = p.take((size_t)S * Bm * gemm_tc_lse_parts(c->ld[t]) * 8);
+  else
+    p.logits = p.take((size_t)S * Bm * c->ld[t] * 4 * (narrow_head(c) ? kHeadSplitsMax : 1));
   p.row_loss = p.take((size_t)S * Bm * 4);
+  p.lse = p.take((size_t)S * Bm * 4);
+  p.label_logit = p.take((size_t)S * Bm * 4);
   p.ev_a = p.take((size_t)Bm * maxN * 4);
   p.ev_b = p.take((size_t)Bm * maxN * 4);
   p.ev_acc = p.take(64);
@@ -396,7 +405,9 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
     auto in_ld = [&](int l) { return l == 0 ? a0_ld : c->ld[l]; };
     auto in_sg = [&](int l) { return l == 0 ? a0_sg : Bm * c->ld[l]; };
 
-    const bool head = narrow_head(c);
+    const bool head = narrow_head(c), wide = wide_head(c);
+    float* lse = c->plan.lse.at<float>(c->ws);
+    float* label_logit = c->plan.label_logit.at<float>(c->ws);
     const int head_ks = head ? gemm_splits(head_splits(c), (int)c->np[t - 1], (const T*)nullptr) : 1;
     // Sec. 2.2: a_l = max((z_l - mean_b z_l) / sigma_b, 0) per subnet and neuron
     auto standardise = [&](int l) {
@@ -433,6 +444,9 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       } else if (l < t) {
         g.epi = EPI_BIAS_RELU;
         g.out = act(l); g.out_ld = c->ld[l]; g.out_sg = Bm * c->ld[l];
+      } else if (wide) {
+        g.epi = EPI_LSE_PART;        // first pass over the output layer: log-sum-exp partials per row
+        g.lse_part = logits;
       } else if (head) {
         g.epi = EPI_BIAS_F32;        // k slices of the logits; bias and the sum happen in the softmax kernel
         g.bias = nullptr;
@@ -451,7 +465,23 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
     // ---- loss and its gradient -------------------------------------------------------------
     {
       Scope sc(c, IST_K_LOSS);
-      if (head)
+      if (wide) {
+        lse_combine(L, logits, gemm_tc_lse_parts(c->ld[t]), S, B, Bm, lse, y + row0, X->stride_subnet, (int)c->N[t], st);
+        GemmArgs<T> g{};             // second pass: the same product, written out as delta_t
+        g.M = B; g.N = (int)c->np[t]; g.K = (int)c->np[t - 1]; g.G = S;
+        g.N_store = (int)c->ld[t];
+        g.A = in_ptr(t - 1); g.a_sm = in_ld(t - 1); g.a_sk = 1; g.a_sg = in_sg(t - 1);
+        g.B = weights(t); g.b_sn = 1; g.b_sk = c->ld[t]; g.b_sg = c->slice_elems(t);
+        g.bias = bias_of(t); g.bias_sg = c->ld[t];
+        g.epi = EPI_SOFTMAX_DELTA;
+        g.out = delta(t); g.out_ld = c->ld[t]; g.out_sg = Bm * c->ld[t];
+        g.lse = lse; g.lse_sg = Bm;
+        g.labels = y + row0; g.labels_sg = X->stride_subnet;
+        g.label_logit = label_logit;
+        g.inv_rows = 1.f / (float)B;
+        if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "softmax pass of the output layer cannot be launched");
+        lse_row_loss(L, lse, label_logit, S, B, Bm, row_loss);
+      } else if (head)
         small_softmax(L, logits, head_ks, c->ld[t], S, B, (int)c->N[t], bias_of(t), c->ld[t], y + row0,
                       X->stride_subnet, delta(t), c->ld[t], Bm * c->ld[t], row_loss, st);
       else

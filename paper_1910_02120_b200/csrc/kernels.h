@@ -62,7 +62,11 @@ enum Epilogue : int {
   EPI_BIAS_F32 = 1,   // outf = C + bias[n]                     (logits)
   EPI_RELU_MASK = 2,  // out = T(mask > 0 ? C : 0)              (delta through ReLU)
   EPI_SGD = 3,        // outf -= lr * C; opw = bf16(outf) if opw (fused weight update)
-  EPI_STORE = 4       // out = T(C)
+  EPI_STORE = 4,      // out = T(C)
+  // Softmax cross-entropy over a very wide output layer without storing the logits (two passes
+  // over the same product):
+  EPI_LSE_PART = 5,   // per row and column tile: (max, sum exp(z - max)) of z = C + bias -> lse_part
+  EPI_SOFTMAX_DELTA = 6  // out = T((exp(z - lse[m]) - [n == label[m]]) * inv_rows); z[m][label[m]] -> label_logit
 };
 
 template <typename T>
@@ -80,12 +84,20 @@ struct GemmArgs {
   const T* mask; int64_t mask_ld, mask_sg;
   bf16* opw;
   float lr;
+  // wide softmax head.  lse_part: [G][2 * ceil(N_store / 256)][M] float2 (two partials per 256-column
+  // tile); lse / label_logit: [G][lse_sg]; labels: labels[g * labels_sg + m].
+  float* lse_part;
+  const float* lse; int64_t lse_sg;
+  const int32_t* labels; int64_t labels_sg;
+  float* label_logit;
+  float inv_rows;
 };
 template <typename T> void gemm_simt(const Launch& L, const GemmArgs<T>& a);
 // Tensor-core path (tcgen05 + TMA) for bf16 operands.  Returns false if the shape cannot be
 // described to TMA (misaligned strides) or the operand layouts do not fit an epilogue.
 bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st);
 int gemm_tc_splits(int K, int want);
+int gemm_tc_lse_parts(int64_t n_store);
 
 // ---- rowops.cu --------------------------------------------------------------------------
 // Row-wise softmax cross-entropy of logits [G][B][ld] against labels; writes
@@ -105,6 +117,13 @@ template <typename T>
 void softmax_xent_small(const Launch& L, const float* part, int ks, int64_t ld, int G, int B, int Nt,
                         const float* bias, int64_t bias_sg, const int32_t* y, int64_t y_sg, T* delta, int64_t ld_d,
                         int64_t sg_d, float* row_loss, DeviceStatus* st);
+// Wide head, between the two passes: lse[g][b] = log sum_n exp(z[g][b][n]) from the per-tile
+// partials ([G][parts][B] float2), labels checked against [0, Nt).  After the second pass:
+// row_loss[g][b] = lse[g][b] - label_logit[g][b].
+void lse_combine(const Launch& L, const float* lse_part, int parts, int G, int B, int64_t lse_sg, float* lse,
+                 const int32_t* y, int64_t y_sg, int Nt, DeviceStatus* st);
+void lse_row_loss(const Launch& L, const float* lse, const float* label_logit, int G, int B, int64_t lse_sg,
+                  float* row_loss);
 // loss_out[g * out_stride + k] = (1/B) sum_b row_loss[g][b]  (fixed summation order)
 void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
                  int64_t out_stride, int k);

@@ -241,6 +241,55 @@ __global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int B, 
   }
 }
 
+// lse[g][b] = log sum_n exp(z[g][b][n]) from per-tile partials (m, s) = (max of z * log2(e),
+// sum of 2^(z * log2(e) - m)).  Block: 32 rows x 32 partial lanes; partials of one index are
+// contiguous over rows.
+__global__ void __launch_bounds__(1024) lse_combine_kernel(const float2* __restrict__ part, int parts, int B,
+                                                            int64_t lse_sg, float* __restrict__ lse,
+                                                            const int32_t* __restrict__ y, int64_t y_sg, int Nt,
+                                                            DeviceStatus* st) {
+  __shared__ float sm[32][33], ss[32][33];
+  pdl_wait();
+  pdl_trigger();
+  const int g = blockIdx.y;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int b = blockIdx.x * 32 + tx;
+  float m = -INFINITY, s = 0.f;
+  if (b < B) {
+    const float2* p = part + (int64_t)g * parts * B + b;
+#pragma unroll 4
+    for (int i = ty; i < parts; i += 32) {
+      const float2 v = p[(int64_t)i * B];
+      if (v.x > -INFINITY) {                       // an empty partial carries (-inf, 0)
+        const float mn = fmaxf(m, v.x);
+        s = s * exp2f(m - mn) + v.y * exp2f(v.x - mn);
+        m = mn;
+      }
+    }
+  }
+  sm[ty][tx] = m;
+  ss[ty][tx] = s;
+  __syncthreads();
+  if (ty == 0 && b < B) {
+    float M = -INFINITY;
+    for (int u = 0; u < 32; ++u) M = fmaxf(M, sm[u][tx]);
+    float S = 0.f;
+    for (int u = 0; u < 32; ++u)
+      if (sm[u][tx] > -INFINITY) S += ss[u][tx] * exp2f(sm[u][tx] - M);
+    lse[(int64_t)g * lse_sg + b] = (M + log2f(S)) * 0.6931471805599453f;
+    const int label = y[(int64_t)g * y_sg + b];
+    if (label < 0 || label >= Nt) report(st, -5, SITE_LABEL, (long long)g * B + b);
+  }
+}
+
+__global__ void lse_row_loss_kernel(const float* __restrict__ lse, const float* __restrict__ zy, int B, int64_t lse_sg,
+                                    float* __restrict__ row_loss) {
+  pdl_wait();
+  pdl_trigger();
+  const int g = blockIdx.y, b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B) row_loss[(int64_t)g * B + b] = lse[(int64_t)g * lse_sg + b] - zy[(int64_t)g * lse_sg + b];
+}
+
 template <typename T>
 __global__ void stage_rows_kernel(const float* __restrict__ X, int64_t N0, int64_t group_row_stride,
                                   int B, T* __restrict__ out, int64_t ld, int64_t sg) {
@@ -380,6 +429,20 @@ template void softmax_xent_small<bf16>(const Launch&, const float*, int, int64_t
 void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
                  int64_t out_stride, int k) {
   launch_pdl(loss_reduce_kernel, dim3(G), dim3(256), 0, L.stream, row_loss, B, loss_out, out_stride, k);
+  L.count();
+}
+
+void lse_combine(const Launch& L, const float* lse_part, int parts, int G, int B, int64_t lse_sg, float* lse,
+                 const int32_t* y, int64_t y_sg, int Nt, DeviceStatus* st) {
+  launch_pdl(lse_combine_kernel, dim3((unsigned)ceil_div(B, 32), G), dim3(1024), 0, L.stream,
+             reinterpret_cast<const float2*>(lse_part), parts, B, lse_sg, lse, y, y_sg, Nt, st);
+  L.count();
+}
+
+void lse_row_loss(const Launch& L, const float* lse, const float* label_logit, int G, int B, int64_t lse_sg,
+                  float* row_loss) {
+  launch_pdl(lse_row_loss_kernel, dim3((unsigned)ceil_div(B, 256), G), dim3(256), 0, L.stream, lse, label_logit, B,
+             lse_sg, row_loss);
   L.count();
 }
 

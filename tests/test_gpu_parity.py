@@ -158,7 +158,8 @@ def test_fp32_round_shapes(dims, S, B, K):
     ([256, 8192, 1000], 8, 512, 2, "normal"),              # large enough for CTA-pair tiles in every GEMM
     ([256, 8192, 8192, 10], 8, 512, 2, "normal"),
     ([264, 6144, 2056, 24], 3, 384, 2, "normal"),          # CTA pairs with ragged edges (M = 384 = 1.5 pair tiles)
-    ([64, 256, 20003], 2, 64, 2, "normal"),                # very wide output: k-split delta GEMM, wide softmax
+    ([64, 256, 20003], 2, 64, 2, "normal"),                # very wide output: k-split delta GEMM, two-pass softmax head
+    ([64, 256, 9001], 2, 160, 2, "normal"),                # the same on CTA pairs, ragged in rows and columns
 ])
 def test_bf16_round_shapes(dims, S, B, K, x_dist):
     _check_round(_wl("b", dims, S, B, K, "bf16", x_dist=x_dist), BF16_W_RTOL, BF16_DW_RTOL,
