@@ -113,12 +113,36 @@ def partition_layer(seed: int, layer: int, N: int, S: int) -> Tuple[np.ndarray, 
     return idx, off
 
 
-def partition(seed: int, layer_dims: Sequence[int], S: int):
+def partition_layer_iid(seed: int, layer: int, N: int, S: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Independent uniform assignment (the other reading of Sec. 2.1 "uniform assignment to one
+    of n possible compute nodes"; App. A: each neuron joins subnet s with probability 1/n,
+    independently of the others): neuron i goes to group floor(key_i * S / 2^64) with the same
+    keys as the balanced rule.  Group sizes are Binomial(N, 1/S), not fixed; a group may be
+    empty.  Indices ascend inside a group.  Returns (idx, off) like partition_layer."""
+    if S < 1 or N < 1:
+        raise ValueError("need S >= 1 and N >= 1")
+    keys = neuron_keys(seed, layer, N)
+    grp = [(int(keys[i]) * S) >> 64 for i in range(N)]
+    idx = np.empty(N, dtype=np.int32)
+    off = np.zeros(S + 1, dtype=np.int32)
+    at = 0
+    for g in range(S):
+        members = [i for i in range(N) if grp[i] == g]      # ascending by construction
+        idx[at:at + len(members)] = members
+        at += len(members)
+        off[g + 1] = at
+    return idx, off
+
+
+PARTITION_RULES = {"balanced": partition_layer, "iid": partition_layer_iid}
+
+
+def partition(seed: int, layer_dims: Sequence[int], S: int, rule: str = "balanced"):
     """One partition per hidden layer l = 1..t-1.  Returns a list of (idx, off)."""
     t = len(layer_dims) - 1
     if t == 1 and S != 1:
         raise ValueError("a network without hidden layers has nothing to partition: S must be 1")
-    return [partition_layer(seed, l, int(layer_dims[l]), S) for l in range(1, t)]
+    return [PARTITION_RULES[rule](seed, l, int(layer_dims[l]), S) for l in range(1, t)]
 
 
 def group(parts, hidden_layer: int, s: int) -> np.ndarray:
@@ -383,7 +407,9 @@ def evaluate(W, b, X, y, dtype=np.float64):
 class IstOracle:
     """partition -> slice -> K local steps per subnet -> copy back."""
 
-    def __init__(self, layer_dims: Sequence[int], S: int, dtype=np.float64, norm_eps=None):
+    def __init__(self, layer_dims: Sequence[int], S: int, dtype=np.float64, norm_eps=None,
+                 partition_rule: str = "balanced"):
+        self.partition_rule = partition_rule
         self.norm_eps = norm_eps          # None: plain path; a float: Sec. 2.2 standardisation
         self.stats = None
         self.layer_dims = [int(d) for d in layer_dims]
@@ -407,7 +433,7 @@ class IstOracle:
         self.b = [np.array(v, dtype=self.dtype, copy=True) for v in b]
 
     def partition(self, seed: int):
-        self.parts = partition(seed, self.layer_dims, self.S)
+        self.parts = partition(seed, self.layer_dims, self.S, self.partition_rule)
         self.subnets = [slice_subnet(self.W, self.b, self.parts, s) for s in range(self.S)]
         return self.parts
 

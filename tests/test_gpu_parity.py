@@ -349,3 +349,25 @@ def test_out_of_range_label_sets_the_device_status():
     assert e.value.status == api.IST_ERR_DEVICE_CHECK
     torch.cuda.synchronize()                   # the context is still usable
     assert torch.isfinite(Wd[0]).all()
+
+
+def _random_shapes(n, seed):
+    g = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        t = int(g.integers(2, 5))
+        S = int(g.integers(1, 7))
+        dims = [int(g.integers(4, 400))] + [int(g.integers(max(S, 8), 700)) for _ in range(t - 1)] + [int(g.integers(2, 300))]
+        out.append((dims, S, int(g.integers(1, 300)), 2))
+    return out
+
+
+@pytest.mark.parametrize("dims,S,B,K", _random_shapes(10, 2024))
+def test_bf16_round_random_shapes(dims, S, B, K):
+    # seeded random widths, subnet counts and batch sizes: ragged tiles in every dimension
+    _check_round(_wl("r", dims, S, B, K, "bf16"), BF16_W_RTOL, BF16_DW_RTOL, BF16_LOSS_ATOL, False)
+
+
+@pytest.mark.parametrize("dims,S,B,K", _random_shapes(6, 77))
+def test_fp32_round_random_shapes(dims, S, B, K):
+    _check_round(_wl("r", dims, S, B, K, "fp32", lr=0.05), FP32_RTOL, 1e-3, FP32_RTOL, True)

@@ -456,3 +456,58 @@ def test_norm_round_and_deployment_statistics():
         ref = _torch_loss_norm([w.detach() for w in tW], [v.detach() for v in tb],
                                torch.tensor(X[0, 0], dtype=torch.float64), torch.tensor(y[0, 0], dtype=torch.long), eps)
     assert abs(ev_loss - ref.item()) < 1e-11
+
+
+# ---------------------------------------------------------------------------------------------
+# independent uniform assignment (the other reading of "uniform assignment", Sec. 2.1 / App. A)
+# ---------------------------------------------------------------------------------------------
+
+def test_iid_partition_is_the_multiply_high_of_the_keys():
+    # brute force with Python integers on the keys (which the published SplitMix64 vector pins)
+    seed, layer, N, S = 99, 2, 257, 5
+    keys = [int(k) for k in O.neuron_keys(seed, layer, N)]
+    idx, off = O.partition_layer_iid(seed, layer, N, S)
+    assert off[0] == 0 and off[-1] == N
+    for g in range(S):
+        want = [i for i in range(N) if (keys[i] * S) // 2 ** 64 == g]
+        assert list(idx[off[g]:off[g + 1]]) == want
+    assert sorted(idx.tolist()) == list(range(N))           # every neuron in exactly one group
+
+
+def test_iid_group_sizes_are_binomial_not_fixed():
+    N, S, trials = 240, 4, 400
+    sizes = np.array([np.diff(O.partition_layer_iid(1000 + s, 1, N, S)[1]) for s in range(trials)])
+    assert sizes.sum(axis=1).tolist() == [N] * trials
+    # mean N/S, variance N (1/S)(1 - 1/S) = 45 per group; the balanced rule would give variance 0
+    assert np.all(np.abs(sizes.mean(axis=0) - N / S) < 4 * np.sqrt(45 / trials))
+    assert np.all(np.abs(sizes.var(axis=0) - 45) < 12)
+    # membership of one neuron is uniform over the groups (chi-square, 3 degrees of freedom)
+    member = np.zeros(S)
+    for s in range(trials):
+        idx, off = O.partition_layer_iid(5000 + s, 1, N, S)
+        member[np.searchsorted(off, np.where(idx == 17)[0][0], side="right") - 1] += 1
+    chi2 = ((member - trials / S) ** 2 / (trials / S)).sum()
+    assert chi2 < 16.3                                       # 0.1 % tail
+
+
+def test_iid_round_reassembles_and_trains_like_the_balanced_one():
+    # slicing and copy-back use only (idx, off): an untouched round is the identity, and with
+    # S = 1 both rules give the same single group and therefore the same trained network
+    dims = [6, 20, 14, 4]
+    W, b, X, y = _tiny(dims, 3, 5, 2)
+    o = O.IstOracle(dims, 3, partition_rule="iid")
+    o.bind_weights(W, b)
+    o.partition(4)
+    sizes = [np.diff(off) for _, off in o.parts]
+    assert any(len(set(s.tolist())) > 1 for s in sizes)     # truly unequal groups for this seed
+    o.reassemble()
+    for l in range(3):
+        assert np.array_equal(o.W[l], W[l].astype(np.float64)) and np.array_equal(o.b[l], b[l].astype(np.float64))
+    W1, b1, X1, y1 = _tiny(dims, 1, 5, 2)
+    a = O.IstOracle(dims, 1, partition_rule="iid")
+    c = O.IstOracle(dims, 1)
+    for o2 in (a, c):
+        o2.bind_weights(W1, b1)
+        o2.round(7, X1, y1, 0.1, 2)
+    for l in range(3):
+        assert np.array_equal(a.W[l], c.W[l])
