@@ -32,6 +32,10 @@ size_t partition_scratch_bytes(int N, int S);
 // Returns false if S is too large for the kernels' shared-memory counters (S > 768).
 bool partition_layer(const Launch& L, uint64_t layer_seed, int N, int S, const PartitionScratch& sc,
                      int32_t* idx, int32_t* off, DeviceStatus* st);
+// Independent uniform assignment: group_i = floor(key_i * S / 2^64); same outputs.
+bool partition_layer_iid(const Launch& L, uint64_t layer_seed, int N, int S, const PartitionScratch& sc, int32_t* idx,
+                         int32_t* off, DeviceStatus* st);
+void partition_iid_counts_host(uint64_t layer_seed, int N, int S, int64_t* counts);
 
 // ---- gather_scatter.cu ------------------------------------------------------------------
 // A slice map describes how packed element (s, i, j) of a layer relates to the full matrix:

@@ -154,7 +154,111 @@ __global__ void emit_kernel(int N, int S, const int32_t* __restrict__ grp, const
   idx[at] = i;
 }
 
+// ---- independent uniform assignment -----------------------------------------------------------
+// group_i = floor(key_i * S / 2^64) with the same keys; group sizes are Binomial(N, 1/S).  The
+// position of a neuron inside its group is found exactly as above (blocks of 1024 neurons in
+// index order); the group offsets come from the block counts instead of a formula.
+__global__ void __launch_bounds__(kPosBlock) iid_group_kernel(uint64_t layer_seed, int N, int S, int32_t* grp,
+                                                               int32_t* lp, int32_t* blkcnt) {
+  extern __shared__ int32_t wcnt[];          // [32 warps][S]
+  const int i = blockIdx.x * kPosBlock + threadIdx.x;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  for (int e = threadIdx.x; e < 32 * S; e += kPosBlock) wcnt[e] = 0;
+  __syncthreads();
+  int g = -1;
+  if (i < N) {
+    const uint64_t k = splitmix64_mix(layer_seed + 0x9E3779B97F4A7C15ull * (uint64_t)(i + 1));
+    g = (int)__umul64hi(k, (uint64_t)S);
+    grp[i] = g;
+  }
+  const unsigned same = __match_any_sync(0xffffffffu, g);
+  const int wpos = __popc(same & ((1u << lane) - 1u));
+  if (g >= 0 && wpos == 0) wcnt[w * S + g] = __popc(same);
+  __syncthreads();
+  if (i < N) {
+    int before = 0;
+    for (int u = 0; u < w; ++u) before += wcnt[u * S + g];
+    lp[i] = before + wpos;
+  }
+  for (int s = threadIdx.x; s < S; s += kPosBlock) {
+    int tot = 0;
+    for (int u = 0; u < 32; ++u) tot += wcnt[u * S + s];
+    blkcnt[(int64_t)blockIdx.x * S + s] = tot;
+  }
+}
+
+// One CTA: off[g] = number of neurons in groups below g.
+__global__ void iid_offsets_kernel(int S, int n_blocks, const int32_t* __restrict__ blkcnt, int32_t* off) {
+  extern __shared__ int32_t tot[];           // [S]
+  for (int s = threadIdx.x; s < S; s += blockDim.x) {
+    int t = 0;
+    for (int u = 0; u < n_blocks; ++u) t += blkcnt[(int64_t)u * S + s];
+    tot[s] = t;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int at = 0;
+    for (int s = 0; s < S; ++s) {
+      off[s] = at;
+      at += tot[s];
+    }
+    off[S] = at;
+  }
+}
+
+__global__ void iid_emit_kernel(int N, int S, const int32_t* __restrict__ grp, const int32_t* __restrict__ lp,
+                                const int32_t* __restrict__ blkcnt, const int32_t* __restrict__ off, int32_t* idx,
+                                DeviceStatus* st) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N) return;
+  const int g = grp[i];
+  if (g < 0 || g >= S) {
+    report(st, -5, SITE_PART_IDX, i);
+    return;
+  }
+  int pos = lp[i];
+  const int blk = i / kPosBlock;
+  for (int u = 0; u < blk; ++u) pos += blkcnt[(int64_t)u * S + g];
+  const int at = off[g] + pos;
+  if (at < off[g] || at >= off[g + 1]) {
+    report(st, -5, SITE_PART_IDX, i);
+    return;
+  }
+  idx[at] = i;
+}
+
 }  // namespace
+
+bool partition_layer_iid(const Launch& L, uint64_t layer_seed, int N, int S, const PartitionScratch& sc, int32_t* idx,
+                         int32_t* off, DeviceStatus* st) {
+  const int smem = 32 * S * (int)sizeof(int32_t);
+  if (smem > 96 * 1024) return false;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(iid_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024) != cudaSuccess)
+      return false;
+    configured = true;
+  }
+  const int n_blocks = (int)ceil_div(N, kPosBlock);
+  iid_group_kernel<<<n_blocks, kPosBlock, smem, L.stream>>>(layer_seed, N, S, sc.grp, sc.lp, sc.blkcnt);
+  iid_offsets_kernel<<<1, 256, S * sizeof(int32_t), L.stream>>>(S, n_blocks, sc.blkcnt, off);
+  iid_emit_kernel<<<(unsigned)ceil_div(N, kThreads), kThreads, 0, L.stream>>>(N, S, sc.grp, sc.lp, sc.blkcnt, off, idx, st);
+  L.count(3);
+  return true;
+}
+
+// Host copy of the same rule: group sizes only (the host needs them to size copies and to refuse
+// a draw that does not fit the packed layout).
+void partition_iid_counts_host(uint64_t layer_seed, int N, int S, int64_t* counts) {
+  for (int s = 0; s < S; ++s) counts[s] = 0;
+  for (int i = 0; i < N; ++i) {
+    uint64_t z = layer_seed + 0x9E3779B97F4A7C15ull * (uint64_t)(i + 1);
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    counts[(int)(((unsigned __int128)z * (unsigned __int128)(uint64_t)S) >> 64)]++;
+  }
+}
 
 size_t partition_scratch_bytes(int N, int S) {
   PartitionScratch s{};
