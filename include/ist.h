@@ -87,6 +87,25 @@ size_t ist_workspace_bytes(const int64_t* layer_dims, int n_dims, int S, int pre
                            int max_batch, int input_is_csr);
 
 /*
+ * The two readings of Sec. 2.1's "uniform assignment to one of n possible compute nodes".
+ * IST_PART_BALANCED (what ist_workspace_bytes / ist_create use): the rule stated at ist_partition,
+ * equal group sizes.  IST_PART_IID: every neuron picks its subnet independently (App. A:
+ * probability 1/n each): group of neuron i = floor(key_i * S / 2^64) with the same keys, indices
+ * ascending inside a group; group sizes are Binomial(N_l, 1/S) and a group may be empty.  The
+ * packed layout then has room for ceil(N_l/S) + ceil(7 * sqrt(N_l (1/S)(1 - 1/S))) + 8 neurons
+ * per subnet and hidden layer (at most N_l); ist_partition returns IST_ERR_UNSUPPORTED, without
+ * enqueueing anything, for a seed whose draw does not fit (probability below 1e-11 per group), and
+ * computes the group sizes on the host (N_l hash evaluations per hidden layer and call).
+ */
+#define IST_PART_BALANCED 0
+#define IST_PART_IID 1
+size_t ist_workspace_bytes2(const int64_t* layer_dims, int n_dims, int S, int precision,
+                            int max_batch, int input_is_csr, int partition_rule);
+ist_status ist_create2(ist_ctx** out, const int64_t* layer_dims, int n_dims, int S, int precision,
+                       int max_batch, int input_is_csr, int partition_rule, void* workspace_dev,
+                       size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Creates a context.  workspace_dev: device, 256-byte aligned, >= ist_workspace_bytes(...).
  * cuda_stream: a cudaStream_t (NULL = legacy default stream), borrowed.  The workspace is
  * cleared on this stream.  *out is set only on success; free it with ist_destroy.

@@ -25,8 +25,9 @@ EXPORTS = [
     "ist_get_subnet_params", "ist_local_steps", "ist_reassemble", "ist_eval", "ist_sync_status",
     "ist_kernel_launches", "ist_last_error", "ist_destroy", "ist_profile", "ist_profile_read",
     "ist_partition_layer_static", "ist_norm_workspace_bytes", "ist_enable_normalization", "ist_calibrate",
-    "ist_set_subnet_range", "ist_packed_layer",
+    "ist_set_subnet_range", "ist_packed_layer", "ist_workspace_bytes2", "ist_create2",
 ]
+IST_PART_BALANCED, IST_PART_IID = 0, 1
 IST_STATIC_MAX_NEURONS, IST_STATIC_MAX_SUBNETS = 65536, 64
 
 KERNEL_CLASSES = ["partition", "gather", "stage", "fwd", "loss", "dx", "dw_sgd", "bias_sgd", "spmm",
@@ -62,6 +63,10 @@ def _load() -> ctypes.CDLL:
     p64 = ctypes.POINTER(ctypes.c_int64)
     lib.ist_workspace_bytes.restype = sz
     lib.ist_workspace_bytes.argtypes = [p64, i32, i32, i32, i32, i32]
+    lib.ist_workspace_bytes2.restype = sz
+    lib.ist_workspace_bytes2.argtypes = [p64, i32, i32, i32, i32, i32, i32]
+    lib.ist_create2.restype = ctypes.c_int32
+    lib.ist_create2.argtypes = [ctypes.POINTER(vp), p64, i32, i32, i32, i32, i32, i32, vp, sz, vp]
     lib.ist_create.restype = ctypes.c_int32
     lib.ist_create.argtypes = [ctypes.POINTER(vp), p64, i32, i32, i32, i32, i32, vp, sz, vp]
     lib.ist_bind_weights.restype = ctypes.c_int32
@@ -123,6 +128,11 @@ def _check(handle, status: int):
         raise IstError(status, lib.ist_last_error(handle).decode())
 
 
+def ist_workspace_bytes2(layer_dims, S, precision, max_batch, input_is_csr=False, partition_rule=0) -> int:
+    arr, n = _dims(layer_dims)
+    return int(lib.ist_workspace_bytes2(arr, n, S, precision, max_batch, int(bool(input_is_csr)), partition_rule))
+
+
 def ist_workspace_bytes(layer_dims, S, precision, max_batch, input_is_csr=False) -> int:
     arr, n = _dims(layer_dims)
     return int(lib.ist_workspace_bytes(arr, n, S, precision, max_batch, int(bool(input_is_csr))))
@@ -174,7 +184,9 @@ class Ist:
     Method names mirror the C calls (ist_partition -> partition, ...)."""
 
     def __init__(self, layer_dims: Sequence[int], S: int, precision: int, max_batch: int,
-                 input_is_csr: bool = False, device: str = "cuda:0", stream: Optional[torch.cuda.Stream] = None):
+                 input_is_csr: bool = False, device: str = "cuda:0", stream: Optional[torch.cuda.Stream] = None,
+                 partition_rule: int = IST_PART_BALANCED):
+        self.partition_rule = int(partition_rule)
         self.layer_dims = [int(d) for d in layer_dims]
         self.t = len(self.layer_dims) - 1
         self.S, self.precision, self.max_batch = int(S), int(precision), int(max_batch)
@@ -182,15 +194,16 @@ class Ist:
         self.device = torch.device(device)
         self.stream = stream
         self.handle = ctypes.c_void_p()
-        nbytes = ist_workspace_bytes(self.layer_dims, S, precision, max_batch, input_is_csr)
+        nbytes = ist_workspace_bytes2(self.layer_dims, S, precision, max_batch, input_is_csr, self.partition_rule)
         if nbytes == 0:
             raise IstError(IST_ERR_ARG, lib.ist_last_error(None).decode())
         self.workspace_bytes = nbytes
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
             arr, n = _dims(self.layer_dims)
-            st = lib.ist_create(ctypes.byref(self.handle), arr, n, self.S, self.precision, self.max_batch,
-                                int(self.input_is_csr), self.workspace.data_ptr(), nbytes, self._stream_ptr())
+            st = lib.ist_create2(ctypes.byref(self.handle), arr, n, self.S, self.precision, self.max_batch,
+                                 int(self.input_is_csr), self.partition_rule, self.workspace.data_ptr(), nbytes,
+                                 self._stream_ptr())
         if st != IST_OK:
             self.handle = ctypes.c_void_p()
             raise IstError(st, lib.ist_last_error(None).decode())
@@ -236,6 +249,9 @@ class Ist:
     def _count(self, l: int, s: int) -> int:
         if l == 0 or l == self.t:
             return self.layer_dims[l]
+        if self.partition_rule == IST_PART_IID:      # sizes vary with the draw: read them back
+            off = self.get_partition(l)[1].cpu()
+            return int(off[s + 1] - off[s])
         N = self.layer_dims[l]
         return N // self.S + (1 if s < N % self.S else 0)
 

@@ -3,6 +3,7 @@
 // of a round runs in this library's kernels; the host only validates and enqueues.
 #include "../../include/ist.h"
 
+#include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <string>
@@ -66,6 +67,10 @@ struct ist_ctx {
   int64_t launches = 0;
   uint64_t seed = 0;
   std::string err;
+
+  // partition rule and, for the independent rule, the group sizes of the partition in place
+  int rule = IST_PART_BALANCED;
+  std::vector<std::vector<int64_t>> group_count;   // [hidden layer][subnet]
 
   // subnets this context trains in ist_local_steps (all S unless ist_set_subnet_range narrowed it)
   int sub_first = 0, sub_count = 0;
@@ -236,7 +241,20 @@ void make_norm_plan(ist_ctx* c) {
   }
 }
 
-void fill_shape(ist_ctx* c, const int64_t* dims, int n_dims, int S, int precision, int max_batch, int csr) {
+// Rows / columns a subnet's slice of a hidden layer is laid out for.  Balanced groups hold
+// ceil(N/S) neurons at most.  Independent assignment gives Binomial(N, 1/S) sizes: the layout has
+// room for the mean plus seven standard deviations (a larger draw, probability < 1e-11 per group,
+// is refused by ist_partition).
+int64_t slice_capacity(int64_t N, int S, int rule) {
+  const int64_t mean = ceil_div(N, (int64_t)S);
+  if (rule != IST_PART_IID || S == 1) return mean;
+  const double sd = std::sqrt((double)N * (1.0 / S) * (1.0 - 1.0 / S));
+  return std::min<int64_t>(N, mean + (int64_t)std::ceil(7.0 * sd) + 8);
+}
+
+void fill_shape(ist_ctx* c, const int64_t* dims, int n_dims, int S, int precision, int max_batch, int csr,
+                int rule = IST_PART_BALANCED) {
+  c->rule = rule;
   c->t = n_dims - 1;
   c->S = S;
   c->sub_first = 0;
@@ -248,7 +266,7 @@ void fill_shape(ist_ctx* c, const int64_t* dims, int n_dims, int S, int precisio
   c->np.resize(n_dims);
   c->ld.resize(n_dims);
   for (int l = 0; l <= c->t; ++l) {
-    c->np[l] = (l == 0 || l == c->t) ? dims[l] : ceil_div(dims[l], S);
+    c->np[l] = (l == 0 || l == c->t) ? dims[l] : slice_capacity(dims[l], S, rule);
     c->ld[l] = round_up(c->np[l], 8);
   }
   make_plan(c);
@@ -555,29 +573,40 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
 
 // ================================= public entry points =======================================
 
-extern "C" size_t ist_workspace_bytes(const int64_t* layer_dims, int n_dims, int S, int precision,
-                                      int max_batch, int input_is_csr) {
+extern "C" size_t ist_workspace_bytes2(const int64_t* layer_dims, int n_dims, int S, int precision,
+                                       int max_batch, int input_is_csr, int partition_rule) {
   std::string why;
   if (!valid_shape(layer_dims, n_dims, S, precision, max_batch, &why)) {
     g_create_error = why;
     return 0;
   }
+  if (partition_rule != IST_PART_BALANCED && partition_rule != IST_PART_IID) {
+    g_create_error = "unknown partition rule";
+    return 0;
+  }
   ist_ctx tmp;
-  fill_shape(&tmp, layer_dims, n_dims, S, precision, max_batch, input_is_csr);
+  fill_shape(&tmp, layer_dims, n_dims, S, precision, max_batch, input_is_csr, partition_rule);
   return tmp.plan.total;
 }
 
-extern "C" ist_status ist_create(ist_ctx** out, const int64_t* layer_dims, int n_dims, int S,
-                                 int precision, int max_batch, int input_is_csr, void* workspace_dev,
-                                 size_t workspace_bytes, void* cuda_stream) {
+extern "C" size_t ist_workspace_bytes(const int64_t* layer_dims, int n_dims, int S, int precision,
+                                      int max_batch, int input_is_csr) {
+  return ist_workspace_bytes2(layer_dims, n_dims, S, precision, max_batch, input_is_csr, IST_PART_BALANCED);
+}
+
+extern "C" ist_status ist_create2(ist_ctx** out, const int64_t* layer_dims, int n_dims, int S,
+                                  int precision, int max_batch, int input_is_csr, int partition_rule,
+                                  void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
   if (!out) return fail(nullptr, IST_ERR_ARG, "out must not be null");
   std::string why;
   if (!valid_shape(layer_dims, n_dims, S, precision, max_batch, &why))
     return fail(nullptr, IST_ERR_ARG, "%s", why.c_str());
+  if (partition_rule != IST_PART_BALANCED && partition_rule != IST_PART_IID)
+    return fail(nullptr, IST_ERR_ARG, "unknown partition rule %d", partition_rule);
   if (input_is_csr && n_dims < 3)
     return fail(nullptr, IST_ERR_UNSUPPORTED, "CSR inputs need at least one hidden layer");
   ist_ctx* c = new ist_ctx();
-  fill_shape(c, layer_dims, n_dims, S, precision, max_batch, input_is_csr);
+  fill_shape(c, layer_dims, n_dims, S, precision, max_batch, input_is_csr, partition_rule);
   if (!workspace_dev || ((uintptr_t)workspace_dev & 255)) {
     delete c;
     return fail(nullptr, IST_ERR_WORKSPACE, "workspace must be a 256-byte aligned device pointer");
@@ -596,6 +625,13 @@ extern "C" ist_status ist_create(ist_ctx** out, const int64_t* layer_dims, int n
   }
   *out = c;
   return IST_OK;
+}
+
+extern "C" ist_status ist_create(ist_ctx** out, const int64_t* layer_dims, int n_dims, int S,
+                                 int precision, int max_batch, int input_is_csr, void* workspace_dev,
+                                 size_t workspace_bytes, void* cuda_stream) {
+  return ist_create2(out, layer_dims, n_dims, S, precision, max_batch, input_is_csr, IST_PART_BALANCED,
+                     workspace_dev, workspace_bytes, cuda_stream);
 }
 
 extern "C" ist_status ist_bind_weights(ist_ctx* c, float* const* W_dev, float* const* b_dev) {
@@ -621,13 +657,30 @@ extern "C" ist_status ist_partition(ist_ctx* c, uint64_t seed) {
   const int t = c->t, S = c->S;
   c->seed = seed;
   uint64_t round_state = seed;
+  if (c->rule == IST_PART_IID) {
+    // group sizes of this draw, from the same rule on the host: nothing is enqueued if a group
+    // does not fit the layout the workspace was sized for
+    uint64_t st = seed;
+    c->group_count.assign(t, std::vector<int64_t>(S, 0));
+    for (int l = 1; l < t; ++l) {
+      const uint64_t layer_seed = splitmix64_next(&st);
+      partition_iid_counts_host(layer_seed, (int)c->N[l], S, c->group_count[l].data());
+      for (int s = 0; s < S; ++s)
+        if (c->group_count[l][s] > c->np[l])
+          return fail(c, IST_ERR_UNSUPPORTED,
+                      "seed %llu puts %lld neurons of hidden layer %d into subnet %d; the layout holds %lld",
+                      (unsigned long long)seed, (long long)c->group_count[l][s], l, s, (long long)c->np[l]);
+    }
+  }
   for (int l = 1; l < t; ++l) {
     Scope sc(c, IST_K_PARTITION);
     uint64_t layer_seed = splitmix64_next(&round_state);
     PartitionScratch ps{};
     partition_scratch_carve(c->plan.part.at<char>(c->ws), (int)c->N[l], S, &ps);
-    if (!partition_layer(L, layer_seed, (int)c->N[l], S, ps, c->idx(l), c->off(l), c->status()))
-      return fail(c, IST_ERR_UNSUPPORTED, "S = %d exceeds what the partition kernels support (768)", S);
+    const bool ok = c->rule == IST_PART_IID
+                        ? partition_layer_iid(L, layer_seed, (int)c->N[l], S, ps, c->idx(l), c->off(l), c->status())
+                        : partition_layer(L, layer_seed, (int)c->N[l], S, ps, c->idx(l), c->off(l), c->status());
+    if (!ok) return fail(c, IST_ERR_UNSUPPORTED, "S = %d exceeds what the partition kernels support (768)", S);
   }
   for (int l = 1; l <= t; ++l) {
     Scope sc(c, IST_K_GATHER);
@@ -660,6 +713,7 @@ extern "C" ist_status ist_get_subnet_params(ist_ctx* c, int layer, int s, float*
   if (layer < 1 || layer > c->t || s < 0 || s >= c->S) return fail(c, IST_ERR_ARG, "layer or subnet out of range");
   auto count = [&](int l) -> int64_t {   // |G_l^s| (balanced split), full width at the ends
     if (l == 0 || l == c->t) return c->N[l];
+    if (c->rule == IST_PART_IID) return c->group_count[l][s];
     return c->N[l] / c->S + (s < c->N[l] % c->S ? 1 : 0);
   };
   Launch L = c->launch();

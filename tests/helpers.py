@@ -32,9 +32,9 @@ def make_problem(w: synth.Workload, bias_scale=0.1, round_index=0):
     return W, b, data
 
 
-def oracle_round(w: synth.Workload, W, b, data, seed, dtype=np.float64, norm_eps=None):
+def oracle_round(w: synth.Workload, W, b, data, seed, dtype=np.float64, norm_eps=None, rule="balanced"):
     from oracle import ist_oracle as O
-    o = O.IstOracle(w.layer_dims, w.S, dtype=dtype, norm_eps=norm_eps)
+    o = O.IstOracle(w.layer_dims, w.S, dtype=dtype, norm_eps=norm_eps, partition_rule=rule)
     o.bind_weights(W, b)
     X = (data.row_ptr, data.col, data.val) if data.is_csr else data.X
     parts = o.partition(seed)
@@ -43,11 +43,12 @@ def oracle_round(w: synth.Workload, W, b, data, seed, dtype=np.float64, norm_eps
     return o, parts, losses
 
 
-def gpu_context(w: synth.Workload, W, b, device="cuda:0"):
+def gpu_context(w: synth.Workload, W, b, device="cuda:0", rule="balanced"):
     import torch
     from paper_1910_02120_b200 import api
     prec = api.IST_BF16 if w.precision == "bf16" else api.IST_FP32
-    ctx = api.Ist(w.layer_dims, w.S, prec, w.B, input_is_csr=(w.x_dist == "csr"), device=device)
+    ctx = api.Ist(w.layer_dims, w.S, prec, w.B, input_is_csr=(w.x_dist == "csr"), device=device,
+                  partition_rule=api.IST_PART_IID if rule == "iid" else api.IST_PART_BALANCED)
     Wd = [torch.tensor(x, device=device) for x in W]
     bd = [torch.tensor(x, device=device) for x in b]
     ctx.bind_weights(Wd, bd)
@@ -70,8 +71,8 @@ def gpu_inputs(w: synth.Workload, data, device="cuda:0", as_bf16=None):
     return X, y
 
 
-def gpu_round(w: synth.Workload, W, b, data, seed, device="cuda:0", as_bf16=None, norm_eps=None):
-    ctx, Wd, bd = gpu_context(w, W, b, device)
+def gpu_round(w: synth.Workload, W, b, data, seed, device="cuda:0", as_bf16=None, norm_eps=None, rule="balanced"):
+    ctx, Wd, bd = gpu_context(w, W, b, device, rule)
     if norm_eps is not None:
         ctx.enable_normalization(norm_eps)
     X, y = gpu_inputs(w, data, device, as_bf16)

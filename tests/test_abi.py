@@ -20,7 +20,7 @@ def api():
 def test_every_declared_symbol_is_exported(api):
     header = open(os.path.join(ROOT, "include", "ist.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(ist_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(ist_[a-z0-9_]+)\s*\(", header))
     assert declared, "no declarations found"
     assert declared == set(api.EXPORTS)
     for name in declared:
