@@ -4,13 +4,14 @@
 //
 // C[g](m, n) = sum_k A[g](m, k) * B[g](n, k) with arbitrary element strides, so the same
 // kernel serves x*W (B is n-contiguous), delta*W^T (B is k-contiguous) and a^T*delta
-// (both operands contiguous along m / n).  64x64 output tile, 16-deep k slabs, 4x4 per thread.
+// (both operands contiguous along m / n).  64x64 output tile (4x4 per thread) or, when that
+// would leave most SMs without a tile, 32x32 (2x2 per thread); 16-deep k slabs.
 #include "kernels.h"
 
 namespace ist {
 namespace {
 
-constexpr int BM = 64, BN = 64, BK = 16, kThreads = 256;
+constexpr int BK = 16, kThreads = 256;
 
 template <typename T>
 __device__ __forceinline__ void epilogue_store(const GemmArgs<T>& a, int g, int m, int n, float c) {
@@ -44,8 +45,9 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs<T>& a, int g, int 
   }
 }
 
-template <typename T>
+template <typename T, int BM, int BN>
 __global__ void __launch_bounds__(kThreads) gemm_simt_kernel(GemmArgs<T> a) {
+  constexpr int TM = BM / 16, TN = BN / 16;      // outputs per thread
   __shared__ float As[BK][BM + 1];
   __shared__ float Bs[BK][BN + 1];
   const int g = blockIdx.z;
@@ -56,47 +58,67 @@ __global__ void __launch_bounds__(kThreads) gemm_simt_kernel(GemmArgs<T> a) {
   const T* B = a.B + (int64_t)g * a.b_sg;
   const bool a_kmajor = a.a_sk == 1, b_kmajor = a.b_sk == 1;
 
-  float acc[4][4];
+  float acc[TM][TN];
 #pragma unroll
-  for (int u = 0; u < 4; ++u)
+  for (int u = 0; u < TM; ++u)
 #pragma unroll
-    for (int v = 0; v < 4; ++v) acc[u][v] = 0.f;
+    for (int v = 0; v < TN; ++v) acc[u][v] = 0.f;
 
-  for (int k0 = 0; k0 < a.K; k0 += BK) {
+  // the next k slab is fetched into registers while the current one is multiplied
+  constexpr int NA = BM * BK / kThreads, NB = BN * BK / kThreads;
+  float ra[NA], rb[NB];
+  auto fetch = [&](int k0) {
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < NA; ++u) {
       int e = tid + kThreads * u;
       int kk = a_kmajor ? e % BK : e / BM;
       int mm = a_kmajor ? e / BK : e % BM;
       int m = m0 + mm, k = k0 + kk;
-      As[kk][mm] = (m < a.M && k < a.K) ? to_float(A[(int64_t)m * a.a_sm + (int64_t)k * a.a_sk]) : 0.f;
-      kk = b_kmajor ? e % BK : e / BN;
+      ra[u] = (m < a.M && k < a.K) ? to_float(A[(int64_t)m * a.a_sm + (int64_t)k * a.a_sk]) : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < NB; ++u) {
+      int e = tid + kThreads * u;
+      int kk = b_kmajor ? e % BK : e / BN;
       int nn = b_kmajor ? e / BK : e % BN;
-      int n = n0 + nn;
-      k = k0 + kk;
-      Bs[kk][nn] = (n < a.N && k < a.K) ? to_float(B[(int64_t)n * a.b_sn + (int64_t)k * a.b_sk]) : 0.f;
+      int n = n0 + nn, k = k0 + kk;
+      rb[u] = (n < a.N && k < a.K) ? to_float(B[(int64_t)n * a.b_sn + (int64_t)k * a.b_sk]) : 0.f;
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < a.K; k0 += BK) {
+#pragma unroll
+    for (int u = 0; u < NA; ++u) {
+      int e = tid + kThreads * u;
+      As[a_kmajor ? e % BK : e / BM][a_kmajor ? e / BK : e % BM] = ra[u];
+    }
+#pragma unroll
+    for (int u = 0; u < NB; ++u) {
+      int e = tid + kThreads * u;
+      Bs[b_kmajor ? e % BK : e / BN][b_kmajor ? e / BK : e % BN] = rb[u];
     }
     __syncthreads();
+    if (k0 + BK < a.K) fetch(k0 + BK);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
-      float av[4], bv[4];
+      float av[TM], bv[TN];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) av[u] = As[kk][ty + 16 * u];
+      for (int u = 0; u < TM; ++u) av[u] = As[kk][ty + 16 * u];
 #pragma unroll
-      for (int v = 0; v < 4; ++v) bv[v] = Bs[kk][tx + 16 * v];
+      for (int v = 0; v < TN; ++v) bv[v] = Bs[kk][tx + 16 * v];
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
+      for (int u = 0; u < TM; ++u)
 #pragma unroll
-        for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(av[u], bv[v], acc[u][v]);
+        for (int v = 0; v < TN; ++v) acc[u][v] = fmaf(av[u], bv[v], acc[u][v]);
     }
     __syncthreads();
   }
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
+  for (int u = 0; u < TM; ++u) {
     int m = m0 + ty + 16 * u;
     if (m >= a.M) continue;
 #pragma unroll
-    for (int v = 0; v < 4; ++v) {
+    for (int v = 0; v < TN; ++v) {
       int n = n0 + tx + 16 * v;
       if (n < a.N) epilogue_store(a, g, m, n, acc[u][v]);
     }
@@ -108,8 +130,15 @@ __global__ void __launch_bounds__(kThreads) gemm_simt_kernel(GemmArgs<T> a) {
 template <typename T>
 void gemm_simt(const Launch& L, const GemmArgs<T>& a) {
   if (a.M <= 0 || a.N <= 0 || a.G <= 0) return;
-  dim3 grid((unsigned)ceil_div(a.N, BN), (unsigned)ceil_div(a.M, BM), (unsigned)a.G);
-  gemm_simt_kernel<T><<<grid, kThreads, 0, L.stream>>>(a);
+  // few large tiles leave most of the 148 SMs idle: use 32x32 tiles until every SM has two
+  const int64_t big = ceil_div(a.N, 64) * ceil_div(a.M, 64) * a.G;
+  if (big >= 296) {
+    dim3 grid((unsigned)ceil_div(a.N, 64), (unsigned)ceil_div(a.M, 64), (unsigned)a.G);
+    gemm_simt_kernel<T, 64, 64><<<grid, kThreads, 0, L.stream>>>(a);
+  } else {
+    dim3 grid((unsigned)ceil_div(a.N, 32), (unsigned)ceil_div(a.M, 32), (unsigned)a.G);
+    gemm_simt_kernel<T, 32, 32><<<grid, kThreads, 0, L.stream>>>(a);
+  }
   L.count();
 }
 
