@@ -44,6 +44,11 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C3", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dims", default="",
+                    help="profiling aid: replace the configuration's layer widths (comma separated); with "
+                         "--subnets / --batch a reduced case of the same kernels for ncu captures")
+    ap.add_argument("--subnets", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--shard-subnets", action="store_true",
                     help="with --gpus N > 1: split the S subnets over the ranks (one all-gather of the trained "
                          "slices per round, strong scaling) instead of running N independent replicas")
@@ -562,6 +567,12 @@ def main():
     w = synth.WORKLOADS[args.config]
     if args.local_steps > 0:
         w = w.scaled(K=args.local_steps, name=w.name + f"-K{args.local_steps}")
+    if args.dims:
+        w = w.scaled(layer_dims=tuple(int(x) for x in args.dims.split(",")), name=w.name + "-reduced")
+    if args.subnets > 0:
+        w = w.scaled(S=args.subnets)
+    if args.batch > 0:
+        w = w.scaled(B=args.batch)
     if args.impl == "reference":
         run_reference(args, w)
     else:
