@@ -65,3 +65,18 @@ def test_normalisation_entry_points_reject_null_contexts(api):
     assert api.lib.ist_norm_workspace_bytes(None) == 0
     assert api.lib.ist_enable_normalization(None, ctypes.c_float(1e-5), None, 0) == api.IST_ERR_ARG
     assert api.lib.ist_calibrate(None, None, 1) == api.IST_ERR_ARG
+
+
+def test_partition_rule_is_validated_and_sizes_the_layout(api):
+    dims = [64, 4096, 4096, 10]
+    bal = api.ist_workspace_bytes2(dims, 8, api.IST_BF16, 128, False, api.IST_PART_BALANCED)
+    iid = api.ist_workspace_bytes2(dims, 8, api.IST_BF16, 128, False, api.IST_PART_IID)
+    assert bal == api.ist_workspace_bytes(dims, 8, api.IST_BF16, 128)
+    assert iid > bal                                  # room for mean + 7 sigma neurons per subnet
+    assert api.ist_workspace_bytes2(dims, 8, api.IST_BF16, 128, False, 7) == 0
+    one_iid = api.ist_workspace_bytes2(dims, 1, api.IST_BF16, 128, False, api.IST_PART_IID)
+    assert one_iid == api.ist_workspace_bytes2(dims, 1, api.IST_BF16, 128, False, api.IST_PART_BALANCED)   # one group holds all
+    dims_c = (ctypes.c_int64 * 3)(8, 4, 3)
+    h = ctypes.c_void_p()
+    st = api.lib.ist_create2(ctypes.byref(h), dims_c, 3, 2, api.IST_FP32, 4, 0, 5, ctypes.c_void_p(256), 1 << 20, None)
+    assert st == api.IST_ERR_ARG and not h.value
