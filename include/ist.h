@@ -24,6 +24,9 @@
  *   - Call order: ist_create -> ist_bind_weights -> { ist_partition -> ist_local_steps* ->
  *     ist_reassemble }* ; ist_eval any time the network is bound and not partitioned.
  *     Between ist_partition and ist_reassemble the caller must not write the bound weights.
+ *   - One process drives one device (kernel attributes and launch limits are looked up once
+ *     per process, on the device current at the first call); several contexts on that device
+ *     are fine, and calls on one context must not overlap in time.
  */
 #ifndef IST_H_
 #define IST_H_
