@@ -15,7 +15,7 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def _sampled_subnet_round(w, s_check, rtol_w, rtol_dw, loss_tol):
+def _sampled_subnet_round(w, s_check, rtol_w, rtol_dw, loss_tol, norm_eps=None, rule="balanced"):
     import torch
     from oracle import ist_oracle as O
     from paper_1910_02120_b200 import api
@@ -23,7 +23,7 @@ def _sampled_subnet_round(w, s_check, rtol_w, rtol_dw, loss_tol):
     W, b = synth.make_weights(w.layer_dims, w.seed)
     data = synth.make_round_inputs(w)
     seed = 31337
-    parts = O.partition(seed, w.layer_dims, w.S)
+    parts = O.partition(seed, w.layer_dims, w.S, rule)
     Ws, bs = O.slice_subnet(W, b, parts, s_check)
     Ws0 = [x.copy() for x in Ws]
     Ws = [x.astype(np.float64) for x in Ws]
@@ -33,13 +33,16 @@ def _sampled_subnet_round(w, s_check, rtol_w, rtol_dw, loss_tol):
     olosses = []
     for k in range(w.K):
         xb, yb = oracle._batch(X, data.y, s_check, k)
-        olosses.append(O.sgd_step(Ws, bs, xb, yb, w.lr))
+        olosses.append(O.sgd_step(Ws, bs, xb, yb, w.lr, norm_eps=norm_eps))
 
     prec = api.IST_BF16 if w.precision == "bf16" else api.IST_FP32
-    ctx = api.Ist(w.layer_dims, w.S, prec, w.B, input_is_csr=data.is_csr, device=dev)
+    ctx = api.Ist(w.layer_dims, w.S, prec, w.B, input_is_csr=data.is_csr, device=dev,
+                  partition_rule=api.IST_PART_IID if rule == "iid" else api.IST_PART_BALANCED)
     Wd = [torch.from_numpy(x).to(dev) for x in W]
     bd = [torch.from_numpy(x).to(dev) for x in b]
     ctx.bind_weights(Wd, bd)
+    if norm_eps is not None:
+        ctx.enable_normalization(norm_eps)
     Xd, yd = H.gpu_inputs(w, data)
     ctx.partition(seed)
     for l in range(1, ctx.t):
@@ -52,8 +55,12 @@ def _sampled_subnet_round(w, s_check, rtol_w, rtol_dw, loss_tol):
         H.assert_close(gw, Ws[l - 1], rtol_w, f"W_{l} of subnet {s_check}")
         # biases start at zero here, so their value is their update: the update tolerance
         # (relative Frobenius error, as for the weight updates) applies
-        fro_b = np.linalg.norm(gb.astype(np.float64) - bs[l - 1]) / max(np.linalg.norm(bs[l - 1]), 1e-300)
-        assert fro_b <= rtol_dw, f"b_{l} of subnet {s_check}: {fro_b:.3e}"
+        if norm_eps is not None and l < ctx.t:
+            # standardisation removes the batch mean: a hidden bias has no gradient and stays (near) zero
+            assert np.max(np.abs(gb)) <= 1e-3 and np.max(np.abs(bs[l - 1])) <= 1e-9
+        else:
+            fro_b = np.linalg.norm(gb.astype(np.float64) - bs[l - 1]) / max(np.linalg.norm(bs[l - 1]), 1e-300)
+            assert fro_b <= rtol_dw, f"b_{l} of subnet {s_check}: {fro_b:.3e}"
         do = Ws[l - 1] - Ws0[l - 1]
         fro = np.linalg.norm((gw.astype(np.float64) - Ws0[l - 1]) - do) / max(np.linalg.norm(do), 1e-300)
         assert fro <= rtol_dw, f"update of W_{l}: {fro:.3e}"
@@ -90,3 +97,16 @@ def test_extreme_classification_config_full_size_one_subnet():
     # wide softmax at their real sizes
     w = synth.C4.scaled(K=1)
     _sampled_subnet_round(w, 1, 2e-2, 1e-1, 5e-3)
+
+
+def test_wide_pixel_config_with_standardisation_one_subnet():
+    # the same shapes with Sec. 2.2's batch standardisation: fp32 pre-activation epilogue on CTA pairs,
+    # column kernels at batch 512
+    w = synth.C3.scaled(K=1)
+    _sampled_subnet_round(w, 3, 2e-2, 1e-1, 5e-3, norm_eps=1e-5)
+
+
+def test_wide_pixel_config_independent_assignment_one_subnet():
+    # unequal groups (capacity-padded slices) at the benchmark's width
+    w = synth.C3.scaled(K=1)
+    _sampled_subnet_round(w, 6, 2e-2, 1e-1, 5e-3, rule="iid")
