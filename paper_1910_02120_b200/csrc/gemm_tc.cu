@@ -138,6 +138,12 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void*
                ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2)
                : "memory");
 }
+// Asks for a box to be brought into L2 only (no shared-memory destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
 __device__ __forceinline__ void tma_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void tma_wait_read() {
@@ -654,6 +660,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           ok = mbar_wait(&slot_empty[slot], ((cq / NS) & 1) ^ 1, abortp, a.status, 6);
           if (!ok) break;
           mbar_expect_tx(&slot_full[slot], AUX_BYTES);
+          if (EPI == EPI_SGD) {
+            // the same chunk of this unit's next tile is asked into L2 now, one tile ahead of its
+            // load, so that the load finds it there; one request per chunk, spread over the tile
+            // (a burst of all of a tile's requests at once measured slower)
+            const int nt = tile + n_units;
+            if (nt < total_tiles) {
+              const int pn = ((nt / a.m_tiles) % a.n_tiles) * BN + c * CH;
+              if (pn < a.N)
+                tma_prefetch_l2_3d(&tmC32, pn, (nt % a.m_tiles) * (BM * PAIR) + rank * BM, nt / (a.m_tiles * a.n_tiles));
+            }
+          }
           if (EPI == EPI_SGD) tma_load_3d(slots + slot * SLOT_BYTES, &tmC32, &slot_full[slot], nc, m0, g);
           else tma_load_3d(slots + slot * SLOT_BYTES + F32_BYTES, &tmAux16, &slot_full[slot], nc, m0, g);
         }
