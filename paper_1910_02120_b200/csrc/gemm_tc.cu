@@ -660,17 +660,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           ok = mbar_wait(&slot_empty[slot], ((cq / NS) & 1) ^ 1, abortp, a.status, 6);
           if (!ok) break;
           mbar_expect_tx(&slot_full[slot], AUX_BYTES);
-          if (EPI == EPI_SGD) {
-            // the same chunk of this unit's next tile is asked into L2 now, one tile ahead of its
-            // load, so that the load finds it there; one request per chunk, spread over the tile
-            // (a burst of all of a tile's requests at once measured slower)
-            const int nt = tile + n_units;
-            if (nt < total_tiles) {
-              const int pn = ((nt / a.m_tiles) % a.n_tiles) * BN + c * CH;
-              if (pn < a.N)
-                tma_prefetch_l2_3d(&tmC32, pn, (nt % a.m_tiles) * (BM * PAIR) + rank * BM, nt / (a.m_tiles * a.n_tiles));
-            }
-          }
           if (EPI == EPI_SGD) tma_load_3d(slots + slot * SLOT_BYTES, &tmC32, &slot_full[slot], nc, m0, g);
           else tma_load_3d(slots + slot * SLOT_BYTES + F32_BYTES, &tmAux16, &slot_full[slot], nc, m0, g);
         }
@@ -705,6 +694,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (ET::k32) tma_store_3d(&tmC32, f32, nc, m0, g);
           if (ET::k16) tma_store_3d(&tmC16, f32 + F32_BYTES, nc, m0, g);
           tma_commit_group();
+          if (EPI == EPI_SGD) {
+            // The same chunk of this unit's next tile is asked into L2 now, one tile ahead of its
+            // load, so that the load finds it there.  The request is issued here, where the
+            // thread would wait for its store anyway; issued by the loader it delayed the loads.
+            const int nt = tile + n_units;
+            if (nt < total_tiles) {
+              const int pn = ((nt / a.m_tiles) % a.n_tiles) * BN + c * CH;
+              if (pn < a.N)
+                tma_prefetch_l2_3d(&tmC32, pn, (nt % a.m_tiles) * (BM * PAIR) + rank * BM, nt / (a.m_tiles * a.n_tiles));
+            }
+          }
           // once the store has read the slot it can be refilled (by the loader) or rewritten (by
           // the epilogue warps); the write to global memory completes in the background
           tma_wait_read<0>();
