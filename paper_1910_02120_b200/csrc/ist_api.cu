@@ -507,7 +507,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
                       X->stride_subnet, delta(t), c->ld[t], Bm * c->ld[t], row_loss, st);
       if (loss_out) loss_reduce(L, row_loss, S, B, loss_out, K, k);
     }
-    // ---- backward + SGD, last layer first.  delta_{l-1} is taken before W_l is updated. -----
+    // ---- backward + SGD, last layer first --------------------------------------------------
     auto update_biases = [&](int l_hi, int l_lo) {   // db_l = sum_b delta_l, layers l_lo..l_hi
       Scope sc(c, IST_K_BIAS_SGD);
       BiasSgdArgs<T> ba{};
@@ -520,8 +520,11 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         }
       }
     };
-    for (int l = t; l >= 1; --l) {
-      if (l > 1) {
+    // Every delta is formed from the weights as they stood at the start of the step, so all of
+    // them are computed first; the bias update follows at once, while the deltas it sums are still
+    // in L2 (after the weight updates have streamed the masters through, they no longer are).
+    for (int l = t; l > 1; --l) {
+      {
         GemmArgs<T> g{};
         g.M = B; g.N = (int)c->np[l - 1]; g.K = (int)c->np[l]; g.G = S;
         g.N_store = (int)c->ld[l - 1];
@@ -531,19 +534,22 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.mask = act(l - 1); g.mask_ld = c->ld[l - 1]; g.mask_sg = Bm * c->ld[l - 1];
         g.out = delta(l - 1); g.out_ld = c->ld[l - 1]; g.out_sg = Bm * c->ld[l - 1];
         Scope sc(c, IST_K_DX);
-        {
         const int want = bf ? wanted_k_splits(c->np[l]) : 1;
         if (want > 1) {
-          if (!split_delta_gemm(c, g, want, B)) return fail(c, IST_ERR_UNSUPPORTED, "k-split delta GEMM of layer %d cannot be launched", l);
-        } else
-        if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMM of layer %d cannot be launched", l);
+          if (!split_delta_gemm(c, g, want, B))
+            return fail(c, IST_ERR_UNSUPPORTED, "k-split delta GEMM of layer %d cannot be launched", l);
+        } else if (!gemm(c, g)) {
+          return fail(c, IST_ERR_UNSUPPORTED, "delta GEMM of layer %d cannot be launched", l);
         }
       }
-      if (l > 1 && c->norm) {   // the masked product is d_zh; carry it through the standardisation
+      if (c->norm) {   // the masked product is d_zh; carry it through the standardisation
         Scope sc(c, IST_K_NORM);
         colnorm_backward<T>(L, delta(l - 1), c->ld[l - 1], Bm * c->ld[l - 1], c->zbuf(l - 1), Bm * c->ld[l - 1],
                             c->nmu(l - 1), c->nrstd(l - 1), c->ld[l - 1], S, B, (int)c->np[l - 1]);
       }
+    }
+    update_biases(t, 1);   // biases are not read by the backward pass
+    for (int l = t; l >= 1; --l) {
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {
         Scope sc(c, IST_K_SPMM);
         spmm_backward_sgd<T>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
@@ -563,7 +569,6 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       Scope sc(c, IST_K_DW_SGD);
       if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "weight-gradient GEMM of layer %d cannot be launched", l);
     }
-    update_biases(t, 1);   // every delta_l is still in place; biases are not read by the backward pass
   }
   IST_CUDA(c, cudaGetLastError());
   return IST_OK;
