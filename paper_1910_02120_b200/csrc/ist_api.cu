@@ -505,17 +505,19 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       else
       softmax_xent<T>(L, logits, c->ld[t], Bm * c->ld[t], S, B, (int)c->N[t], y + row0,
                       X->stride_subnet, delta(t), c->ld[t], Bm * c->ld[t], row_loss, st);
-      if (loss_out) loss_reduce(L, row_loss, S, B, loss_out, K, k);
     }
     // ---- backward + SGD, last layer first --------------------------------------------------
-    auto update_biases = [&](int l_hi, int l_lo) {   // db_l = sum_b delta_l, layers l_lo..l_hi
+    // db_l = sum_b delta_l, layers l_lo..l_hi; the step's mean losses are reduced by the same launch
+    auto update_biases = [&](int l_hi, int l_lo) {
       Scope sc(c, IST_K_BIAS_SGD);
       BiasSgdArgs<T> ba{};
+      LossReduce lo{row_loss, loss_out, K, k};
       int n = 0;
       for (int l = l_hi; l >= l_lo; --l) {
         ba.layer[n++] = BiasSgdLayer<T>{delta(l), c->ld[l], Bm * c->ld[l], bias_of(l), c->ld[l], (int)c->np[l]};
         if (n == kMaxBiasLayers || l == l_lo) {
-          bias_sgd<T>(L, ba, n, S, B, lr);
+          bias_sgd<T>(L, ba, n, S, B, lr, lo);
+          lo.loss_out = nullptr;
           n = 0;
         }
       }

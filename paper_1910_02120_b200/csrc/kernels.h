@@ -128,11 +128,17 @@ void lse_combine(const Launch& L, const float* lse_part, int parts, int G, int B
                  const int32_t* y, int64_t y_sg, int Nt, DeviceStatus* st);
 void lse_row_loss(const Launch& L, const float* lse, const float* label_logit, int G, int B, int64_t lse_sg,
                   float* row_loss);
-// loss_out[g * out_stride + k] = (1/B) sum_b row_loss[g][b]  (fixed summation order)
-void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
-                 int64_t out_stride, int k);
+// loss_out[g * out_stride + k] = (1/B) sum_b row_loss[g][b]  (fixed summation order); rides on
+// the bias update's launch (see bias_sgd) so that it costs no launch of its own.
+struct LossReduce {
+  const float* row_loss;   // [G][B]
+  float* loss_out;         // null: no loss wanted
+  int64_t out_stride;
+  int k;
+};
 // bias[g][n] -= lr * sum_b delta[g][b][n] for up to kMaxBiasLayers layers in one launch.
-// delta rows are ld elements long (ld a multiple of 8, 16-byte aligned); n <= ld.
+// delta rows are ld elements long (ld a multiple of 8, 16-byte aligned); n <= ld.  If
+// loss.loss_out is set, G extra blocks of the same launch reduce the step's row losses.
 constexpr int kMaxBiasLayers = 8;
 template <typename T> struct BiasSgdLayer {
   const T* delta; int64_t ld, sg;
@@ -141,7 +147,7 @@ template <typename T> struct BiasSgdLayer {
 };
 template <typename T> struct BiasSgdArgs { BiasSgdLayer<T> layer[kMaxBiasLayers]; };
 template <typename T>
-void bias_sgd(const Launch& L, const BiasSgdArgs<T>& a, int n_layers, int G, int B, float lr);
+void bias_sgd(const Launch& L, const BiasSgdArgs<T>& a, int n_layers, int G, int B, float lr, const LossReduce& loss);
 // fp32 rows -> T rows with leading dimension ld (pad columns zero), per group row offsets.
 template <typename T>
 void stage_rows(const Launch& L, const float* X, int64_t N0, int64_t group_row_stride, int G, int B,

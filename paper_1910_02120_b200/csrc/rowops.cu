@@ -180,20 +180,9 @@ __global__ void __launch_bounds__(256) softmax_xent_small_kernel(
   if (lane == 0) row_loss[(int64_t)g * B + b] = logf(se) + mx - zl;
 }
 
-__global__ void loss_reduce_kernel(const float* __restrict__ row_loss, int B, float* loss_out,
-                                   int64_t out_stride, int k) {
-  __shared__ float sh[32];
-  pdl_wait();
-  pdl_trigger();
-  int g = blockIdx.x;
-  float acc = 0.f;
-  for (int b = threadIdx.x; b < B; b += blockDim.x) acc += row_loss[(int64_t)g * B + b];
-  acc = block_sum(acc, sh);
-  if (threadIdx.x == 0) loss_out[(int64_t)g * out_stride + k] = acc / (float)B;
-}
-
 // Bias gradient and update of every layer in one launch: blockIdx.z = layer, blockIdx.y = group,
-// blockIdx.x = block of 64 columns.  Thread (cx, ry) sums 8 adjacent columns over rows
+// blockIdx.x = block of 64 columns.  One more z-plane, when a loss is wanted, holds one block per
+// group that averages the step's row losses (256 threads, fixed summation order).  Thread (cx, ry) sums 8 adjacent columns over rows
 // ry, ry + 32, ...; the 32 partial sums of a column are added in a fixed order.
 __device__ __forceinline__ void load8(const float* p, float v[8]) {
   float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
@@ -207,10 +196,19 @@ __device__ __forceinline__ void load8(const bf16* p, float v[8]) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int B, float lr) {
+__global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int n_layers, int B, float lr, LossReduce lo) {
   __shared__ float part[32][65];
   pdl_wait();
   pdl_trigger();
+  if ((int)blockIdx.z == n_layers) {
+    if (blockIdx.x != 0) return;
+    const int g = blockIdx.y;
+    float acc = 0.f;
+    for (int b = threadIdx.x; b < B; b += blockDim.x) acc += lo.row_loss[(int64_t)g * B + b];
+    acc = block_sum(acc, &part[0][0]);
+    if (threadIdx.x == 0) lo.loss_out[(int64_t)g * lo.out_stride + lo.k] = acc / (float)B;
+    return;
+  }
   const BiasSgdLayer<T> L = a.layer[blockIdx.z];
   const int g = blockIdx.y;
   const int cx = threadIdx.x & 7, ry = threadIdx.x >> 3;
@@ -426,12 +424,6 @@ void softmax_xent_small(const Launch& L, const float* part, int ks, int64_t ld, 
 template void softmax_xent_small<bf16>(const Launch&, const float*, int, int64_t, int, int, int, const float*, int64_t,
                                        const int32_t*, int64_t, bf16*, int64_t, int64_t, float*, DeviceStatus*);
 
-void loss_reduce(const Launch& L, const float* row_loss, int G, int B, float* loss_out,
-                 int64_t out_stride, int k) {
-  launch_pdl(loss_reduce_kernel, dim3(G), dim3(256), 0, L.stream, row_loss, B, loss_out, out_stride, k);
-  L.count();
-}
-
 void lse_combine(const Launch& L, const float* lse_part, int parts, int G, int B, int64_t lse_sg, float* lse,
                  const int32_t* y, int64_t y_sg, int Nt, DeviceStatus* st) {
   launch_pdl(lse_combine_kernel, dim3((unsigned)ceil_div(B, 32), G), dim3(1024), 0, L.stream,
@@ -447,14 +439,15 @@ void lse_row_loss(const Launch& L, const float* lse, const float* label_logit, i
 }
 
 template <typename T>
-void bias_sgd(const Launch& L, const BiasSgdArgs<T>& a, int n_layers, int G, int B, float lr) {
-  int64_t max_ld = 0;
+void bias_sgd(const Launch& L, const BiasSgdArgs<T>& a, int n_layers, int G, int B, float lr, const LossReduce& loss) {
+  int64_t max_ld = 64;
   for (int i = 0; i < n_layers; ++i) max_ld = a.layer[i].ld > max_ld ? a.layer[i].ld : max_ld;
-  launch_pdl(bias_sgd_kernel<T>, dim3((unsigned)ceil_div(max_ld, 64), G, n_layers), dim3(256), 0, L.stream, a, B, lr);
+  launch_pdl(bias_sgd_kernel<T>, dim3((unsigned)ceil_div(max_ld, 64), G, n_layers + (loss.loss_out ? 1 : 0)), dim3(256), 0,
+             L.stream, a, n_layers, B, lr, loss);
   L.count();
 }
-template void bias_sgd<float>(const Launch&, const BiasSgdArgs<float>&, int, int, int, float);
-template void bias_sgd<bf16>(const Launch&, const BiasSgdArgs<bf16>&, int, int, int, float);
+template void bias_sgd<float>(const Launch&, const BiasSgdArgs<float>&, int, int, int, float, const LossReduce&);
+template void bias_sgd<bf16>(const Launch&, const BiasSgdArgs<bf16>&, int, int, int, float, const LossReduce&);
 
 template <typename T>
 void stage_rows(const Launch& L, const float* X, int64_t N0, int64_t group_row_stride, int G, int B,
