@@ -509,6 +509,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int c = 0; c < NCH; ++c, ++cq) {
         const int nc = n0 + c * CH;
         if (nc >= a.N) break;                         // CTA-uniform
+        // A slot always belongs to the same warp group, so that the group sees the slot's barrier
+        // phases in order (a parity wait cannot tell phase p from phase p + 2); every configuration
+        // that stores through the ring has an even number of slots, so the groups alternate.
+        static_assert(!kStore || NS % 2 == 0, "slot ring needs an even number of slots");
         if ((cq & 1) != wg) continue;
         const int slot = cq % NS;
         uint8_t* f32 = slots + slot * SLOT_BYTES;
@@ -931,10 +935,10 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
     case EPI_BIAS_RELU:
       if (a_mn || !b_mn) return false;
       if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
-      if (pair == 2) return launch<0, 1, 256, 6, 3, EPI_BIAS_RELU, 2>(L, m, t);
-      if (bn == 256) return launch<0, 1, 256, 4, 3, EPI_BIAS_RELU, 1>(L, m, t);
-      if (bn == 128) return launch<0, 1, 128, 6, 3, EPI_BIAS_RELU, 1>(L, m, t);
-      return launch<0, 1, 64, 8, 3, EPI_BIAS_RELU, 1>(L, m, t);
+      if (pair == 2) return launch<0, 1, 256, 6, 4, EPI_BIAS_RELU, 2>(L, m, t);
+      if (bn == 256) return launch<0, 1, 256, 4, 4, EPI_BIAS_RELU, 1>(L, m, t);
+      if (bn == 128) return launch<0, 1, 128, 6, 4, EPI_BIAS_RELU, 1>(L, m, t);
+      return launch<0, 1, 64, 8, 4, EPI_BIAS_RELU, 1>(L, m, t);
     case EPI_BIAS_F32:
       if (a_mn) return false;
       if (!make_map(&m.c32, a.outf, 4, n_store, a.M, (long long)a.G * t.k_splits, a.outf_ld, a.outf_sg, CH, BM, 128))
@@ -942,16 +946,16 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
       if (!a_mn && !b_mn) {   // both operands K-major: k slices of delta * W^T
         if (pair == 2) return launch<0, 0, 256, 6, 2, EPI_BIAS_F32, 2>(L, m, t);
         if (bn == 256) return launch<0, 0, 256, 4, 2, EPI_BIAS_F32, 1>(L, m, t);
-        if (bn == 128) return launch<0, 0, 128, 5, 3, EPI_BIAS_F32, 1>(L, m, t);
-        return launch<0, 0, 64, 6, 3, EPI_BIAS_F32, 1>(L, m, t);
+        if (bn == 128) return launch<0, 0, 128, 5, 4, EPI_BIAS_F32, 1>(L, m, t);
+        return launch<0, 0, 64, 6, 4, EPI_BIAS_F32, 1>(L, m, t);
       }
       // a short contraction (wide output layer fed by a narrow hidden layer) is bound by writing
       // the logits: fewer operand stages, a deeper ring of output chunks
       if (pair == 2 && ceil_div(a.K, BK) <= 4) return launch<0, 1, 256, 3, 6, EPI_BIAS_F32, 2>(L, m, t);
       if (pair == 2) return launch<0, 1, 256, 6, 2, EPI_BIAS_F32, 2>(L, m, t);
       if (bn == 256) return launch<0, 1, 256, 4, 2, EPI_BIAS_F32, 1>(L, m, t);
-      if (bn == 128) return launch<0, 1, 128, 5, 3, EPI_BIAS_F32, 1>(L, m, t);
-      return launch<0, 1, 64, 6, 3, EPI_BIAS_F32, 1>(L, m, t);
+      if (bn == 128) return launch<0, 1, 128, 5, 4, EPI_BIAS_F32, 1>(L, m, t);
+      return launch<0, 1, 64, 6, 4, EPI_BIAS_F32, 1>(L, m, t);
     case EPI_LSE_PART:
       if (a_mn || !b_mn || a.k_splits > 1 || !a.lse_part) return false;
       if (pair == 2) return launch<0, 1, 256, 4, 1, EPI_LSE_PART, 2>(L, m, t);
