@@ -698,7 +698,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (ET::k32) tma_store_3d(&tmC32, f32, nc, m0, g);
           if (ET::k16) tma_store_3d(&tmC16, f32 + F32_BYTES, nc, m0, g);
           tma_commit_group();
-          if (EPI == EPI_SGD) {
+          if (EPI == EPI_SGD && PAIR == 2) {
             // The same chunk of this unit's next tile is asked into L2 now, one tile ahead of its
             // load, so that the load finds it there.  The request is issued here, where the
             // thread would wait for its store anyway; issued by the loader it delayed the loads.

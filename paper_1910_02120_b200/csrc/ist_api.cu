@@ -377,6 +377,8 @@ void small_softmax(const Launch& L, const float* part, int ks, int64_t ld, int G
                    float* row_loss, DeviceStatus* st) {
   softmax_xent_small<bf16>(L, part, ks, ld, G, B, Nt, bias, bias_sg, y, y_sg, delta, ld_d, sg_d, row_loss, st);
 }
+// Working sets up to this size are taken to survive in the 126 MB L2 between two kernels.
+constexpr size_t kL2ResidentBytes = 64u << 20;
 // One call of ist_local_steps in operand type T.
 template <typename T>
 ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, float lr, int K,
@@ -550,7 +552,12 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
                             c->nmu(l - 1), c->nrstd(l - 1), c->ld[l - 1], S, B, (int)c->np[l - 1]);
       }
     }
-    update_biases(t, 1);   // biases are not read by the backward pass
+    // biases are not read by the backward pass, so their update may come before or after the
+    // weight updates: before, if the deltas it sums are small enough to be still in L2 then
+    size_t delta_bytes = 0;
+    for (int l = 1; l <= t; ++l) delta_bytes += (size_t)S * B * c->ld[l] * sizeof(T);
+    const bool bias_first = delta_bytes <= kL2ResidentBytes;
+    if (bias_first) update_biases(t, 1);
     for (int l = t; l >= 1; --l) {
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {
         Scope sc(c, IST_K_SPMM);
@@ -571,6 +578,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       Scope sc(c, IST_K_DW_SGD);
       if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "weight-gradient GEMM of layer %d cannot be launched", l);
     }
+    if (!bias_first) update_biases(t, 1);
   }
   IST_CUDA(c, cudaGetLastError());
   return IST_OK;

@@ -145,7 +145,10 @@ template <typename T> struct BiasSgdLayer {
   float* bias; int64_t bias_sg;
   int n;
 };
-template <typename T> struct BiasSgdArgs { BiasSgdLayer<T> layer[kMaxBiasLayers]; };
+template <typename T> struct BiasSgdArgs {
+  BiasSgdLayer<T> layer[kMaxBiasLayers];
+  int xstart[kMaxBiasLayers + 1];   // filled in by bias_sgd: first block of each layer
+};
 template <typename T>
 void bias_sgd(const Launch& L, const BiasSgdArgs<T>& a, int n_layers, int G, int B, float lr, const LossReduce& loss);
 // fp32 rows -> T rows with leading dimension ld (pad columns zero), per group row offsets.

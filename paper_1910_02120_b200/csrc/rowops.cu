@@ -180,10 +180,12 @@ __global__ void __launch_bounds__(256) softmax_xent_small_kernel(
   if (lane == 0) row_loss[(int64_t)g * B + b] = logf(se) + mx - zl;
 }
 
-// Bias gradient and update of every layer in one launch: blockIdx.z = layer, blockIdx.y = group,
-// blockIdx.x = block of 64 columns.  One more z-plane, when a loss is wanted, holds one block per
-// group that averages the step's row losses (256 threads, fixed summation order).  Thread (cx, ry) sums 8 adjacent columns over rows
-// ry, ry + 32, ...; the 32 partial sums of a column are added in a fixed order.
+// Bias gradient and update of every layer in one launch: blockIdx.y = group, blockIdx.x runs over
+// the layers' blocks of 64 columns one layer after the other (layer i owns blocks xstart[i] ..
+// xstart[i + 1] - 1).  Thread (cx, ry) sums 8 adjacent columns over rows ry, ry + 32, ...; the 32
+// partial sums of a column are added in a fixed order.  When a loss is wanted the grid has one
+// more column of blocks (one per group) that averages the step's row losses (256 threads, fixed
+// summation order).
 __device__ __forceinline__ void load8(const float* p, float v[8]) {
   float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
   v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
@@ -200,8 +202,7 @@ __global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int n_l
   __shared__ float part[32][65];
   pdl_wait();
   pdl_trigger();
-  if ((int)blockIdx.z == n_layers) {
-    if (blockIdx.x != 0) return;
+  if ((int)blockIdx.x == a.xstart[n_layers]) {   // the extra column of blocks
     const int g = blockIdx.y;
     float acc = 0.f;
     for (int b = threadIdx.x; b < B; b += blockDim.x) acc += lo.row_loss[(int64_t)g * B + b];
@@ -209,11 +210,12 @@ __global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int n_l
     if (threadIdx.x == 0) lo.loss_out[(int64_t)g * lo.out_stride + lo.k] = acc / (float)B;
     return;
   }
-  const BiasSgdLayer<T> L = a.layer[blockIdx.z];
-  const int g = blockIdx.y;
+  int li = 0;
+  while (li + 1 < n_layers && (int)blockIdx.x >= a.xstart[li + 1]) ++li;
+  const BiasSgdLayer<T> L = a.layer[li];
+  const int g = blockIdx.y, bx = blockIdx.x - a.xstart[li];
   const int cx = threadIdx.x & 7, ry = threadIdx.x >> 3;
-  const int c0 = blockIdx.x * 64 + cx * 8;
-  if (blockIdx.x * 64 >= L.ld) return;
+  const int c0 = bx * 64 + cx * 8;
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (c0 < L.ld) {
     const T* d = L.delta + (int64_t)g * L.sg + c0;
@@ -229,7 +231,7 @@ __global__ void __launch_bounds__(256) bias_sgd_kernel(BiasSgdArgs<T> a, int n_l
   for (int e = 0; e < 8; ++e) part[ry][cx * 8 + e] = acc[e];
   __syncthreads();
   if (threadIdx.x < 64) {
-    const int col = blockIdx.x * 64 + threadIdx.x;
+    const int col = bx * 64 + threadIdx.x;
     if (col < L.n) {
       float s = 0.f;
 #pragma unroll
@@ -440,10 +442,11 @@ void lse_row_loss(const Launch& L, const float* lse, const float* label_logit, i
 
 template <typename T>
 void bias_sgd(const Launch& L, const BiasSgdArgs<T>& a, int n_layers, int G, int B, float lr, const LossReduce& loss) {
-  int64_t max_ld = 64;
-  for (int i = 0; i < n_layers; ++i) max_ld = a.layer[i].ld > max_ld ? a.layer[i].ld : max_ld;
-  launch_pdl(bias_sgd_kernel<T>, dim3((unsigned)ceil_div(max_ld, 64), G, n_layers + (loss.loss_out ? 1 : 0)), dim3(256), 0,
-             L.stream, a, n_layers, B, lr, loss);
+  BiasSgdArgs<T> b = a;
+  b.xstart[0] = 0;
+  for (int i = 0; i < n_layers; ++i) b.xstart[i + 1] = b.xstart[i] + (int)ceil_div(a.layer[i].ld, 64);
+  launch_pdl(bias_sgd_kernel<T>, dim3((unsigned)b.xstart[n_layers] + (loss.loss_out ? 1 : 0), G), dim3(256), 0, L.stream, b,
+             n_layers, B, lr, loss);
   L.count();
 }
 template void bias_sgd<float>(const Launch&, const BiasSgdArgs<float>&, int, int, int, float, const LossReduce&);
