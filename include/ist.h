@@ -230,6 +230,18 @@ ist_status ist_calibrate(ist_ctx* ctx, const ist_input* X, int64_t n);
 ist_status ist_sync_status(ist_ctx* ctx);
 
 /*
+ * Self-test of the device-side error path (no counterpart in the paper).  Every wait inside the
+ * tensor-core kernels is bounded: after its limit it records IST_ERR_DEVICE_TIMEOUT in the status
+ * word and the kernel returns.  This call enqueues, on the context's stream, a one-block kernel that
+ * waits with the same routine on a barrier nothing ever signals, for limit_cycles SM clock cycles
+ * (1 .. 2e9, i.e. at most about a second), so that the wait must give up.  Afterwards
+ * ist_sync_status returns IST_ERR_DEVICE_TIMEOUT for this context (the status word is sticky: create
+ * a new context to go on); the stream and the device stay usable.  Returns IST_ERR_ARG for a limit
+ * outside the range, IST_ERR_CUDA if the launch fails.
+ */
+ist_status ist_selftest_wait_expiry(ist_ctx* ctx, int64_t limit_cycles);
+
+/*
  * Measurement aid (no counterpart in the paper).  Kernel classes of a round, in the order a
  * round runs them.  With profiling enabled every group of launches of one class is bracketed
  * by a pair of CUDA events on the context's stream; ist_profile_read synchronises and returns

@@ -26,6 +26,7 @@ EXPORTS = [
     "ist_kernel_launches", "ist_last_error", "ist_destroy", "ist_profile", "ist_profile_read",
     "ist_partition_layer_static", "ist_norm_workspace_bytes", "ist_enable_normalization", "ist_calibrate",
     "ist_set_subnet_range", "ist_packed_layer", "ist_workspace_bytes2", "ist_create2",
+    "ist_selftest_wait_expiry",
 ]
 IST_PART_BALANCED, IST_PART_IID = 0, 1
 IST_STATIC_MAX_NEURONS, IST_STATIC_MAX_SUBNETS = 65536, 64
@@ -85,6 +86,8 @@ def _load() -> ctypes.CDLL:
     lib.ist_eval.argtypes = [vp, ctypes.POINTER(IstInput), vp, i64, vp, vp]
     lib.ist_sync_status.restype = ctypes.c_int32
     lib.ist_sync_status.argtypes = [vp]
+    lib.ist_selftest_wait_expiry.restype = ctypes.c_int32
+    lib.ist_selftest_wait_expiry.argtypes = [vp, i64]
     lib.ist_kernel_launches.restype = i64
     lib.ist_kernel_launches.argtypes = [vp]
     lib.ist_last_error.restype = ctypes.c_char_p
@@ -321,6 +324,11 @@ class Ist:
 
     def sync_status(self):
         _check(self.handle, lib.ist_sync_status(self.handle))
+
+    def selftest_wait_expiry(self, limit_cycles: int):
+        """Enqueues a kernel whose bounded wait must expire; sync_status() then raises with
+        IST_ERR_DEVICE_TIMEOUT."""
+        _check(self.handle, lib.ist_selftest_wait_expiry(self.handle, int(limit_cycles)))
 
     def profile(self, enable: bool):
         _check(self.handle, lib.ist_profile(self.handle, int(bool(enable))))

@@ -86,13 +86,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  Returns false (and raises the abort flag) if the phase did not complete in time
 // or another role has already aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          DeviceStatus* st, int where) {
+                                          DeviceStatus* st, int where, long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = clock64();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (clock64() - t0 > limit_cycles) {
       *abort_flag = 1;
       report(st, -6, SITE_TC_PIPE, where);
       return false;
@@ -702,6 +702,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // The same chunk of this unit's next tile is asked into L2 now, one tile ahead of its
             // load, so that the load finds it there.  The request is issued here, where the
             // thread would wait for its store anyway; issued by the loader it delayed the loads.
+            // Only on CTA pairs: with single-CTA tiles (short contractions over slices one tile
+            // high) the requests measured slower than going without.
             const int nt = tile + n_units;
             if (nt < total_tiles) {
               const int pn = ((nt / a.m_tiles) % a.n_tiles) * BN + c * CH;
@@ -730,6 +732,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
                    : "memory");
   }
+}
+
+// Self-test of the bounded wait: one thread waits on a barrier that nothing ever signals, with
+// the given limit, so the wait has to give up, record the status and return.  where = 99.
+__global__ void wait_expiry_kernel(DeviceStatus* st, long long limit_cycles) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(&bar, 0, &abort_flag, st, 99, limit_cycles);
+  __syncthreads();
 }
 
 // ---- host side ---------------------------------------------------------------------------------
@@ -860,6 +877,12 @@ bool launch(const Launch& L, const Maps& m, const TcArgs& t) {
 }
 
 }  // namespace
+
+bool gemm_tc_wait_selftest(const Launch& L, DeviceStatus* st, long long limit_cycles) {
+  wait_expiry_kernel<<<1, 32, 0, L.stream>>>(st, limit_cycles);
+  L.count();
+  return cudaGetLastError() == cudaSuccess;
+}
 
 // Tile shape.  Pairs of CTAs (256 x 256 tiles) are used when the problem has enough of them to
 // give every SM pair work; otherwise single CTAs with the widest of 256 / 128 / 64 columns that

@@ -923,6 +923,15 @@ extern "C" ist_status ist_sync_status(ist_ctx* c) {
   return IST_OK;
 }
 
+extern "C" ist_status ist_selftest_wait_expiry(ist_ctx* c, int64_t limit_cycles) {
+  if (!c) return IST_ERR_ARG;
+  if (limit_cycles < 1 || limit_cycles > 2000000000ll)
+    return fail(c, IST_ERR_ARG, "limit_cycles must be in 1..2e9 (about a second)");
+  if (!gemm_tc_wait_selftest(c->launch(), c->status(), limit_cycles))
+    return fail(c, IST_ERR_CUDA, "the self-test kernel could not be launched");
+  return IST_OK;
+}
+
 extern "C" ist_status ist_profile(ist_ctx* c, int enable) {
   if (!c) return IST_ERR_ARG;
   IST_CUDA(c, cudaStreamSynchronize(c->stream));

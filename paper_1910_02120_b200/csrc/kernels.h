@@ -100,6 +100,9 @@ template <typename T> void gemm_simt(const Launch& L, const GemmArgs<T>& a);
 // Tensor-core path (tcgen05 + TMA) for bf16 operands.  Returns false if the shape cannot be
 // described to TMA (misaligned strides) or the operand layouts do not fit an epilogue.
 bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st);
+// Launches a one-block kernel whose bounded barrier wait must expire after limit_cycles (see
+// ist_selftest_wait_expiry).
+bool gemm_tc_wait_selftest(const Launch& L, DeviceStatus* st, long long limit_cycles);
 int gemm_tc_splits(int K, int want);
 int gemm_tc_lse_parts(int64_t n_store);
 
