@@ -144,6 +144,10 @@ __device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int c
                ::"l"(map), "r"(c0), "r"(c1), "r"(c2)
                : "memory");
 }
+// Brings a tensor map (a kernel parameter) into the descriptor cache ahead of its first copy.
+__device__ __forceinline__ void prefetch_map(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
 __device__ __forceinline__ void tma_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void tma_wait_read() {
@@ -309,6 +313,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int rank = PAIR == 2 ? (int)cluster_ctarank() : 0;
   const int unit = blockIdx.x / PAIR, n_units = gridDim.x / PAIR;   // a unit = a CTA or a pair
 
+  if (threadIdx.x == 32) {   // the maps this instance copies through; they do not depend on the previous kernel
+    prefetch_map(&tmA);
+    prefetch_map(&tmB);
+    if (ET::k32) prefetch_map(&tmC32);
+    if (ET::k16) prefetch_map(&tmC16);
+    if (EPI == EPI_RELU_MASK) prefetch_map(&tmAux16);
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(&full_bar[s], 1);
