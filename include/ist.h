@@ -26,7 +26,8 @@
  *     Between ist_partition and ist_reassemble the caller must not write the bound weights.
  *   - One process drives one device (kernel attributes and launch limits are looked up once
  *     per process, on the device current at the first call); several contexts on that device
- *     are fine, and calls on one context must not overlap in time.
+ *     are fine, and calls on one context must not overlap in time.  Calls may come from any
+ *     host thread, including one that has made no CUDA call before.
  */
 #ifndef IST_H_
 #define IST_H_

@@ -816,6 +816,11 @@ bool make_map(CUtensorMap* out, const void* base, int elem_bytes, long long inne
   }
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
+  // The encoder is a driver call and wants the device's context current on the calling thread; a
+  // thread that has made no runtime call yet has none (the launches that follow would bind it, but
+  // they come after this).
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaSetDevice(dev) != cudaSuccess) return false;
   cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)groups};
   cuuint64_t strides[2] = {(cuuint64_t)outer_stride * elem_bytes,
                            (cuuint64_t)(groups > 1 ? group_stride : outer_stride * outer) * elem_bytes};
