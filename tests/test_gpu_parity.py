@@ -142,6 +142,8 @@ def test_fp32_round_tiny_config():
     ([64, 256, 256, 35], 4, 64, 5),
     ([40, 301, 10], 3, 8, 2),            # first layer wide enough for the staged column permutation, odd width
     ([16, 2500, 6], 5, 4, 1),            # more than one staged column chunk
+    ([32] + [64] * 10 + [10], 2, 16, 2), # eleven layers: the bias update takes more than one launch
+    ([16, 8, 8, 4], 8, 8, 2),            # one neuron per group
 ])
 def test_fp32_round_shapes(dims, S, B, K):
     _check_round(_wl("s", dims, S, B, K, "fp32", lr=0.05), FP32_RTOL, 1e-3, FP32_RTOL, True)
@@ -160,6 +162,9 @@ def test_fp32_round_shapes(dims, S, B, K):
     ([264, 6144, 2056, 24], 3, 384, 2, "normal"),          # CTA pairs with ragged edges (M = 384 = 1.5 pair tiles)
     ([64, 256, 20003], 2, 64, 2, "normal"),                # very wide output: k-split delta GEMM, two-pass softmax head
     ([64, 256, 9001], 2, 160, 2, "normal"),                # the same on CTA pairs, ragged in rows and columns
+    ([64, 256, 128, 10], 2, 700, 2, "normal"),             # batch larger than 512
+    ([16, 8, 8, 4], 8, 8, 2, "normal"),                    # one neuron per group
+    ([64, 256, 8192], 2, 64, 2, "normal"),                 # widest output layer that still stores its logits
 ])
 def test_bf16_round_shapes(dims, S, B, K, x_dist):
     _check_round(_wl("b", dims, S, B, K, "bf16", x_dist=x_dist), BF16_W_RTOL, BF16_DW_RTOL,
