@@ -38,6 +38,8 @@ def test_iid_partition_matches_oracle_bit_exact(dims, S):
     ("fp32", [20, 37, 5], 3, 7, 3),
     ("fp32", [33, 129, 65, 130, 11], 4, 33, 2),
     ("bf16", [256, 1024, 1024, 35], 4, 256, 3),
+    ("fp32", [16, 10, 9, 4], 8, 8, 2),             # nearly as many subnets as neurons: some groups are empty
+    ("bf16", [16, 10, 9, 4], 8, 8, 2),
     ("bf16", [48, 515, 300, 10], 5, 24, 2),
     ("bf16", [256, 8192, 1000], 8, 512, 2),
 ])

@@ -146,3 +146,16 @@ def test_calibrate_then_eval_matches_oracle(csr):
     ctx.reassemble()
     with pytest.raises(api.IstError):
         ctx.eval(Xg, torch.tensor(y, device="cuda:0"), n)
+
+
+def test_standardisation_with_independent_assignment():
+    # both optional modes at once: Binomial group sizes and batch statistics over padded slices
+    w = _wl([64, 256, 128, 10], 4, 64, 2, "bf16", lr=0.01)
+    W, b, data = H.make_problem(w, bias_scale=0.1)
+    o, oparts, oloss = H.oracle_round(w, W, b, data, 7, norm_eps=EPS, rule="iid")
+    ctx, gW, gb, gparts, gloss = H.gpu_round(w, W, b, data, 7, norm_eps=EPS, rule="iid")
+    for (gi, go), (oi, oo) in zip(gparts, oparts):
+        assert np.array_equal(gi, oi) and np.array_equal(go, oo)
+    assert abs(gloss.mean() - oloss.mean()) <= BF16_LOSS_ATOL
+    for l in range(len(W)):
+        H.assert_close(gW[l], o.W[l], BF16_W_RTOL, f"W_{l + 1}")
