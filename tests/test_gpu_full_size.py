@@ -110,3 +110,58 @@ def test_wide_pixel_config_independent_assignment_one_subnet():
     # unequal groups (capacity-padded slices) at the benchmark's width
     w = synth.C3.scaled(K=1)
     _sampled_subnet_round(w, 6, 2e-2, 1e-1, 5e-3, rule="iid")
+
+
+def test_largest_sweep_width_indexes_beyond_two_to_the_31():
+    """1024 -> 65536 -> 65536 -> 100 with two subnets: the middle layer has 2^32 entries, every
+    subnet owns 2^30 of them.  No CPU run can follow that, so the round is checked through what holds
+    at any size: with lr = 0 it returns the network bit for bit; with lr > 0 no entry outside a
+    subnet's own block moves and nearly all inside do."""
+    import torch
+    from paper_1910_02120_b200 import api
+    dev = "cuda:0"
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70 * 2**30:
+        pytest.skip("needs about 70 GB of device memory")
+    Hw, S, B = 65536, 2, 512
+    dims = (1024, Hw, Hw, 100)
+    g = torch.Generator(device=dev)
+    g.manual_seed(3)
+    Wd = [torch.empty(dims[i], dims[i + 1], device=dev).uniform_(-0.01, 0.01, generator=g) for i in range(3)]
+    bd = [torch.zeros(dims[i + 1], device=dev) for i in range(3)]
+    ref = [w.clone() for w in Wd]
+    X = torch.randn(S * B, dims[0], device=dev, generator=g).to(torch.bfloat16)
+    y = torch.randint(0, 100, (S * B,), device=dev, dtype=torch.int32, generator=g)
+    ctx = api.Ist(dims, S, api.IST_BF16, B, device=dev)
+    ctx.bind_weights(Wd, bd)
+    ctx.partition(11)
+    (idx1, off1), (idx2, off2) = ctx.get_partition(1), ctx.get_partition(2)
+    losses = ctx.local_steps(X, y, 0.0, 1, B)
+    ctx.reassemble()
+    ctx.sync_status()
+    assert all(torch.equal(a, r) for a, r in zip(Wd, ref))
+    assert torch.isfinite(losses).all() and (losses > 4.0).all() and (losses < 5.2).all()   # ln 100 = 4.6
+
+    ctx.partition(11)
+    ctx.local_steps(X, y, 0.5, 1, B)
+    ctx.reassemble()
+    ctx.sync_status()
+    grp1 = torch.empty(Hw, dtype=torch.int64, device=dev)
+    grp2 = torch.empty(Hw, dtype=torch.int64, device=dev)
+    for s in range(S):
+        grp1[idx1[off1[s]:off1[s + 1]].long()] = s
+        grp2[idx2[off2[s]:off2[s + 1]].long()] = s
+    moved_outside = moved_inside = inside = 0
+    for r0 in range(0, Hw, 4096):
+        moved = Wd[1][r0:r0 + 4096] != ref[1][r0:r0 + 4096]
+        own = grp1[r0:r0 + 4096, None] == grp2[None, :]
+        moved_outside += int((moved & ~own).sum())
+        moved_inside += int((moved & own).sum())
+        inside += int(own.sum())
+    assert inside == Hw * Hw // S
+    assert moved_outside == 0
+    assert moved_inside > 0.99 * inside
+    assert int((Wd[1][-1] != ref[1][-1]).sum()) > 0.99 * Hw // S                    # the last row is reached
+    assert int((Wd[0] != ref[0]).sum()) > 0.99 * Wd[0].numel()
+    del ctx, Wd, ref
+    torch.cuda.empty_cache()
