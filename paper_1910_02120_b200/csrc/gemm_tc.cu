@@ -57,6 +57,7 @@ constexpr int kEpiWarps = 8;
 constexpr int kAuxWarp = 10;
 constexpr int kStoreWarp0 = 11, kStoreWarps = 4;
 constexpr long long kWaitLimitCycles = 2000000000ll;   // ~1 s at 2 GHz
+constexpr uint32_t kSuspendHintNs = 20000;             // a waiting thread may sleep this long inside one try_wait
 
 // ---- small PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -76,10 +77,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs)
       : "memory");
   return ok != 0;
 }
