@@ -84,14 +84,15 @@ typedef struct ist_input {
 /*
  * Bytes of device workspace a context of this shape needs (0 on invalid arguments).
  * layer_dims: host, n_dims = t+1 entries, each >= 1.  S >= 1 subnets (S = 1 if t = 1),
- * S <= every hidden N_l.  max_batch >= 1: largest `batch` later passed in ist_input
+ * S <= every hidden N_l.  1 <= max_batch <= 65535: largest `batch` later passed in ist_input
  * (ist_eval processes its rows in chunks of max_batch).
  */
 size_t ist_workspace_bytes(const int64_t* layer_dims, int n_dims, int S, int precision,
                            int max_batch, int input_is_csr);
 
 /*
- * The two readings of Sec. 2.1's "uniform assignment to one of n possible compute nodes".
+ * Sec. 2.1 "Constructing Subnets" says only that each hidden neuron is assigned uniformly at
+ * random to one of the n sites; it does not say whether group sizes are fixed.  Two readings:
  * IST_PART_BALANCED (what ist_workspace_bytes / ist_create use): the rule stated at ist_partition,
  * equal group sizes.  IST_PART_IID: every neuron picks its subnet independently (App. A:
  * probability 1/n each): group of neuron i = floor(key_i * S / 2^64) with the same keys, indices
@@ -110,7 +111,10 @@ ist_status ist_create2(ist_ctx** out, const int64_t* layer_dims, int n_dims, int
                        size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Creates a context.  workspace_dev: device, 256-byte aligned, >= ist_workspace_bytes(...).
+ * Creates a context for a network of the paper's form (Sec. 2: an input layer, t - 1 hidden
+ * layers and an output layer with weight matrices between consecutive layers, trained at n = S
+ * sites).  Contexts and workspaces themselves have no counterpart in the paper.
+ * workspace_dev: device, 256-byte aligned, >= ist_workspace_bytes(...).
  * cuda_stream: a cudaStream_t (NULL = legacy default stream), borrowed.  The workspace is
  * cleared on this stream.  *out is set only on success; free it with ist_destroy.
  */
@@ -119,7 +123,8 @@ ist_status ist_create(ist_ctx** out, const int64_t* layer_dims, int n_dims, int 
                       void* cuda_stream);
 
 /*
- * The full network the rounds act on.  W_dev / b_dev: host arrays of t device pointers
+ * The full network the rounds act on (Sec. 2.1: the model the subnets are cut from and copied
+ * back into).  W_dev / b_dev: host arrays of t device pointers
  * (W_l [N_{l-1}][N_l] fp32, b_l [N_l] fp32), borrowed until ist_destroy or the next bind.
  */
 ist_status ist_bind_weights(ist_ctx* ctx, float* const* W_dev, float* const* b_dev);
@@ -129,8 +134,9 @@ ist_status ist_bind_weights(ist_ctx* ctx, float* const* W_dev, float* const* b_d
  * every hidden layer from `seed` and gathers each subnet's slices into the workspace:
  * subnet s owns W_1[:, G_1^s], W_l[G_{l-1}^s, G_l^s] for 1 < l < t, W_t[G_{t-1}^s, :], the
  * hidden biases of its neurons and its own copy of the output bias (App. A: each neuron in
- * exactly one subnet; footnote: inactive neurons are never computed).
- * Partition rule (the paper states only "uniform assignment"): neuron i of hidden layer l
+ * exactly one subnet; its footnote: a subnet's weight slices leave out everything that belongs
+ * to neurons the subnet does not own).
+ * Partition rule (the paper states only that the assignment is uniform): neuron i of hidden layer l
  * gets the i-th output of a SplitMix64 generator seeded with the l-th output of a SplitMix64
  * generator seeded with `seed`; neurons are ranked by (key, index); group g takes the next
  * floor(N_l/S) (+1 if g < N_l mod S) ranks; indices are ascending inside a group.
@@ -138,7 +144,8 @@ ist_status ist_bind_weights(ist_ctx* ctx, float* const* W_dev, float* const* b_d
 ist_status ist_partition(ist_ctx* ctx, uint64_t seed);
 
 /*
- * Copies the current partition of hidden layer `hidden_layer` (1..t-1) out:
+ * Copies the current partition of hidden layer `hidden_layer` (1..t-1) out, i.e. the membership
+ * indicators of App. A as index lists (group s = the neurons j with m^(s)_{l,j} = 1):
  * idx_out_dev [N_l] int32 (group-major, ascending inside a group), off_out_dev [S+1] int32.
  */
 ist_status ist_get_partition(ist_ctx* ctx, int hidden_layer, int32_t* idx_out_dev,
@@ -153,6 +160,15 @@ ist_status ist_get_subnet_params(ist_ctx* ctx, int layer, int s, float* W_out_de
                                  float* b_out_dev);
 
 /*
+ * Shape of subnet s's slice of layer l (1..t) under the partition in place (Sec. 2.1; Sec. 2.3
+ * counts these sizes): *rows_out_host = |G_{l-1}^s| (N_0 for l = 1), *cols_out_host = |G_l^s|
+ * (N_t for l = t).  Host outputs, either may be NULL.  These are the extents
+ * ist_get_subnet_params writes.  Needs a partition in place (IST_ERR_STATE otherwise).
+ */
+ist_status ist_subnet_slice_shape(ist_ctx* ctx, int layer, int s, int64_t* rows_out_host,
+                                  int64_t* cols_out_host);
+
+/*
  * Sec. 2.1 "Training Subnets": K iterations of local SGD on every subnet, no exchange.
  * Step k of subnet s: forward (App. A Eq. (2) on the slice, without the n^2 factor, as
  * Sec. 2.2 removes it), mean softmax cross-entropy against y, backward, w <- w - lr * grad
@@ -165,16 +181,17 @@ ist_status ist_local_steps(ist_ctx* ctx, const ist_input* X, const int32_t* y_de
                            float* loss_out_dev);
 
 /*
- * Training the S subnets at several sites (Sec. 2.1: "Each of the n subnets is sent to a compute
- * node"; Sec. 2.3: only the slices travel).  A context may train only subnets first .. first +
- * count - 1 in ist_local_steps; the other subnets' slices are trained by other contexts (other
- * GPUs, one process each) that hold a copy of the same full network and draw the same
- * partition (same seed).  Before ist_reassemble every context must hold all S trained slices:
- * ist_packed_layer gives the device address of layer l's packed fp32 slices
- * ([S][*master_bytes_per_subnet], subnet s at byte offset s * bytes) and of its packed biases,
- * so that the caller can exchange them (one all-gather per layer over the subnet dimension, each
- * site contributing its own `count` slabs).  ist_partition still gathers all S slices and
- * ist_reassemble still writes all S back; only ist_local_steps is narrowed.
+ * Training the S subnets at several sites (Sec. 2.1 "Distributing Subnets": every subnet goes to
+ * its own compute node; Sec. 2.3: only the slices travel).  A context may own only subnets
+ * first .. first + count - 1: ist_partition then draws the whole partition (it is cheap and every
+ * site needs the same one) but gathers only the owned subnets' slices, and ist_local_steps trains
+ * only those; the other subnets are trained by other contexts (other GPUs, one process each) that
+ * hold a copy of the same full network and draw the same partition (same seed).  Before
+ * ist_reassemble every context must hold all S trained slices: ist_packed_layer gives the device
+ * address of layer l's packed fp32 slices ([S][*master_bytes_per_subnet], subnet s at byte
+ * offset s * bytes) and of its packed biases, so that the caller can exchange them (one
+ * all-gather per layer over the subnet dimension, each site contributing its own `count` slabs).
+ * ist_reassemble writes all S slabs back, whoever trained them.
  * In ist_local_steps the inputs and losses are then addressed by the local subnet index
  * (0 .. count-1): rows start at i * stride_subnet, loss_out_dev holds count * K values.
  * Default range: all S subnets.  Not allowed while a partition is in place.
@@ -184,7 +201,8 @@ ist_status ist_packed_layer(ist_ctx* ctx, int layer, void** master_dev, size_t* 
                             void** bias_dev, size_t* bias_bytes_per_subnet);
 
 /*
- * Sec. 2.1: "subnet parameters are copied back into the full NN, where no collisions occur".
+ * Sec. 2.1 "Training Subnets", last step: the trained slices go back into the full network; the
+ * groups are disjoint, so no two subnets write the same entry.
  * Writes every trained slice to the positions it was gathered from; entries of middle layers
  * whose row group differs from their column group are not written.  The output bias, the one
  * parameter all subnets hold, becomes b + (sum_s (b^(s) - b)) / S (its mean over the copies).
@@ -300,6 +318,17 @@ ist_status ist_profile_read(ist_ctx* ctx, int kernel_class, int64_t* launches_ou
 #define IST_STATIC_MAX_SUBNETS 64
 ist_status ist_partition_layer_static(uint64_t seed, int hidden_layer, int64_t n_neurons, int S,
                                       int32_t* idx_out_dev, int32_t* off_out_dev, void* cuda_stream);
+
+/*
+ * Device-side status of ist_partition_layer_static on the current device (no counterpart in the
+ * paper).  Its kernels check every index they emit against [0, n_neurons) and record a failure
+ * in a status word at the start of the built-in array; each call of the entry point clears the
+ * word first, so this reports on the most recent call.  Waits for cuda_stream (the stream that
+ * call used), copies the word to the host and returns IST_OK or IST_ERR_DEVICE_CHECK
+ * (IST_ERR_CUDA if the copy fails).  Allocates nothing.  Before the first
+ * ist_partition_layer_static call on the device it returns IST_OK.
+ */
+ist_status ist_static_partition_status(void* cuda_stream);
 
 /* Number of kernels this context has launched so far (host counter). */
 int64_t ist_kernel_launches(const ist_ctx* ctx);

@@ -18,8 +18,9 @@ What follows the paper, and what is a reading of it where the paper is silent:
   independently per layer; input and output neurons belong to every subnet.
   READING (group sizes are never stated): a balanced random split, see
   `partition_layer`.
-* Sec. 2.1, App. A footnote ("inactive neurons are never computed"): subnet s
-  owns W_l[G_{l-1}^s, G_l^s]; first layer sliced on columns only, last layer on
+* Sec. 2.1, App. A footnote (weights are cut so that nothing belonging to a
+  neuron outside the subnet is ever evaluated): subnet s owns
+  W_l[G_{l-1}^s, G_l^s]; first layer sliced on columns only, last layer on
   rows only.
 * App. A Eq. (2) with the n^2 factor removed, as Sec. 2.2 "Correcting
   Distributional Shift" does: f_l = S(W_l f_{l-1}) on the slice, scale 1.

@@ -26,7 +26,7 @@ EXPORTS = [
     "ist_kernel_launches", "ist_last_error", "ist_destroy", "ist_profile", "ist_profile_read",
     "ist_partition_layer_static", "ist_norm_workspace_bytes", "ist_enable_normalization", "ist_calibrate",
     "ist_set_subnet_range", "ist_packed_layer", "ist_workspace_bytes2", "ist_create2",
-    "ist_selftest_wait_expiry",
+    "ist_selftest_wait_expiry", "ist_subnet_slice_shape", "ist_static_partition_status",
 ]
 IST_PART_BALANCED, IST_PART_IID = 0, 1
 IST_STATIC_MAX_NEURONS, IST_STATIC_MAX_SUBNETS = 65536, 64
@@ -78,6 +78,10 @@ def _load() -> ctypes.CDLL:
     lib.ist_get_partition.argtypes = [vp, i32, vp, vp]
     lib.ist_get_subnet_params.restype = ctypes.c_int32
     lib.ist_get_subnet_params.argtypes = [vp, i32, i32, vp, vp]
+    lib.ist_subnet_slice_shape.restype = ctypes.c_int32
+    lib.ist_subnet_slice_shape.argtypes = [vp, i32, i32, p64, p64]
+    lib.ist_static_partition_status.restype = ctypes.c_int32
+    lib.ist_static_partition_status.argtypes = [vp]
     lib.ist_local_steps.restype = ctypes.c_int32
     lib.ist_local_steps.argtypes = [vp, ctypes.POINTER(IstInput), vp, ctypes.c_float, i32, vp]
     lib.ist_reassemble.restype = ctypes.c_int32
@@ -181,6 +185,15 @@ def ist_partition_layer_static(seed: int, hidden_layer: int, n_neurons: int, S: 
                                                   ctypes.c_void_p(s.cuda_stream)))
 
 
+def ist_static_partition_status(stream: Optional[torch.cuda.Stream] = None, device=None) -> int:
+    """Waits for `stream` and returns the device status word of ist_partition_layer_static's kernels
+    on the current device (IST_OK unless one of their bounds checks tripped)."""
+    dev = torch.device(device) if device is not None else torch.device("cuda", torch.cuda.current_device())
+    with torch.cuda.device(dev):
+        s = stream if stream is not None else torch.cuda.current_stream(dev)
+        return int(lib.ist_static_partition_status(ctypes.c_void_p(s.cuda_stream)))
+
+
 class Ist:
     """One IST context: owns the workspace tensor, borrows the full network's tensors.
 
@@ -249,18 +262,16 @@ class Ist:
         _check(self.handle, lib.ist_get_partition(self.handle, hidden_layer, idx.data_ptr(), off.data_ptr()))
         return idx, off
 
-    def _count(self, l: int, s: int) -> int:
-        if l == 0 or l == self.t:
-            return self.layer_dims[l]
-        if self.partition_rule == IST_PART_IID:      # sizes vary with the draw: read them back
-            off = self.get_partition(l)[1].cpu()
-            return int(off[s + 1] - off[s])
-        N = self.layer_dims[l]
-        return N // self.S + (1 if s < N % self.S else 0)
+    def subnet_slice_shape(self, layer: int, s: int) -> Tuple[int, int]:
+        """(rows, cols) of subnet s's slice of layer `layer` under the partition in place."""
+        rows, cols = ctypes.c_int64(), ctypes.c_int64()
+        _check(self.handle, lib.ist_subnet_slice_shape(self.handle, layer, s, ctypes.byref(rows), ctypes.byref(cols)))
+        return int(rows.value), int(cols.value)
 
     def get_subnet_params(self, layer: int, s: int):
-        Wt = torch.empty((self._count(layer - 1, s), self._count(layer, s)), dtype=torch.float32, device=self.device)
-        bt = torch.empty(self._count(layer, s), dtype=torch.float32, device=self.device)
+        rows, cols = self.subnet_slice_shape(layer, s)
+        Wt = torch.empty((rows, cols), dtype=torch.float32, device=self.device)
+        bt = torch.empty(cols, dtype=torch.float32, device=self.device)
         _check(self.handle, lib.ist_get_subnet_params(self.handle, layer, s, Wt.data_ptr(), bt.data_ptr()))
         return Wt, bt
 

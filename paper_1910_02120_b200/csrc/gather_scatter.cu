@@ -1,7 +1,11 @@
 // Partition-indexed gather / scatter of weight slices between the full network and the
-// per-subnet packed buffers (paper Sec. 2.1: weights are "partitioned accordingly based on the
-// active neurons"; "subnet parameters are copied back into the full NN").  Pure data movement:
+// per-subnet packed buffers (paper Sec. 2.1 "Constructing Subnets": a subnet's weights are the
+// entries whose row and column neurons it owns; "Training Subnets": the trained slices go back
+// to the positions they came from).  Pure data movement:
 // fp32 values are moved bit for bit; the bf16 operand copy is a rounding of the moved value.
+#include <algorithm>
+#include <mutex>
+
 #include "kernels.h"
 
 namespace ist {
@@ -15,49 +19,52 @@ constexpr int kRowsPerCta = 8;
 // neurons stay inert through the local steps.
 __global__ void gather_kernel(const float* __restrict__ W, SliceMap m, float* __restrict__ master,
                               bf16* __restrict__ opw) {
-  int s = blockIdx.z;
+  int s = m.s_first + blockIdx.z;
   int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (j >= m.ld) return;
   int64_t ncols = m.col_idx ? (m.col_off[s + 1] - m.col_off[s]) : m.full_cols;
   int64_t nrows = m.row_idx ? (m.row_off[s + 1] - m.row_off[s]) : m.full_rows;
   int64_t c = -1;
   if (j < ncols) c = m.col_idx ? m.col_idx[m.col_off[s] + j] : j;
-  int64_t i0 = (int64_t)blockIdx.y * kRowsPerCta;
-  float v[kRowsPerCta];
+  // row blocks blockIdx.y, blockIdx.y + gridDim.y, ... (the y dimension of a grid stops at 65535)
+  for (int64_t i0 = (int64_t)blockIdx.y * kRowsPerCta; i0 < m.rows_pad; i0 += (int64_t)gridDim.y * kRowsPerCta) {
+    float v[kRowsPerCta];
 #pragma unroll
-  for (int u = 0; u < kRowsPerCta; ++u) {
-    int64_t i = i0 + u;
-    v[u] = 0.f;
-    if (c >= 0 && i < nrows) {
-      int64_t r = m.row_idx ? m.row_idx[m.row_off[s] + i] : i;
-      v[u] = __ldg(W + r * m.full_cols + c);
+    for (int u = 0; u < kRowsPerCta; ++u) {
+      int64_t i = i0 + u;
+      v[u] = 0.f;
+      if (c >= 0 && i < nrows) {
+        int64_t r = m.row_idx ? m.row_idx[m.row_off[s] + i] : i;
+        v[u] = __ldg(W + r * m.full_cols + c);
+      }
     }
-  }
 #pragma unroll
-  for (int u = 0; u < kRowsPerCta; ++u) {
-    int64_t i = i0 + u;
-    if (i < m.rows_pad) {
-      int64_t o = ((int64_t)s * m.rows_pad + i) * m.ld + j;
-      master[o] = v[u];
-      if (opw) opw[o] = __float2bfloat16_rn(v[u]);
+    for (int u = 0; u < kRowsPerCta; ++u) {
+      int64_t i = i0 + u;
+      if (i < m.rows_pad) {
+        int64_t o = ((int64_t)s * m.rows_pad + i) * m.ld + j;
+        master[o] = v[u];
+        if (opw) opw[o] = __float2bfloat16_rn(v[u]);
+      }
     }
   }
 }
 
 __global__ void scatter_kernel(float* __restrict__ W, SliceMap m, const float* __restrict__ master) {
-  int s = blockIdx.z;
+  int s = m.s_first + blockIdx.z;
   int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   int64_t ncols = m.col_idx ? (m.col_off[s + 1] - m.col_off[s]) : m.full_cols;
   int64_t nrows = m.row_idx ? (m.row_off[s + 1] - m.row_off[s]) : m.full_rows;
   if (j >= ncols) return;
   int64_t c = m.col_idx ? m.col_idx[m.col_off[s] + j] : j;
-  int64_t i0 = (int64_t)blockIdx.y * kRowsPerCta;
+  for (int64_t i0 = (int64_t)blockIdx.y * kRowsPerCta; i0 < nrows; i0 += (int64_t)gridDim.y * kRowsPerCta) {
 #pragma unroll
-  for (int u = 0; u < kRowsPerCta; ++u) {
-    int64_t i = i0 + u;
-    if (i < nrows) {
-      int64_t r = m.row_idx ? m.row_idx[m.row_off[s] + i] : i;
-      W[r * m.full_cols + c] = master[((int64_t)s * m.rows_pad + i) * m.ld + j];
+    for (int u = 0; u < kRowsPerCta; ++u) {
+      int64_t i = i0 + u;
+      if (i < nrows) {
+        int64_t r = m.row_idx ? m.row_idx[m.row_off[s] + i] : i;
+        W[r * m.full_cols + c] = master[((int64_t)s * m.rows_pad + i) * m.ld + j];
+      }
     }
   }
 }
@@ -72,7 +79,7 @@ constexpr int kStageRows = 8;
 constexpr int kStageCols = 2048;
 constexpr int kMaxGroupsStaged = 64;
 
-struct ColRuns {                 // per group: packed positions [lo, lo + cnt) fall in the chunk
+struct ColRuns {                 // per group moved (m.s_first + i): packed positions [lo, lo + cnt) fall in the chunk
   int lo[kMaxGroupsStaged];
   int pre[kMaxGroupsStaged + 1]; // prefix sums of cnt
 };
@@ -89,12 +96,12 @@ __device__ __forceinline__ int lower_bound_idx(const int32_t* idx, int n, int c)
 
 __device__ __forceinline__ void find_runs(const SliceMap& m, int S, int c0, int c1, ColRuns* runs) {
   if (threadIdx.x < S) {
-    const int s = threadIdx.x;
+    const int s = m.s_first + threadIdx.x;
     const int32_t* g = m.col_idx + m.col_off[s];
     const int n = m.col_off[s + 1] - m.col_off[s];
     const int lo = lower_bound_idx(g, n, c0);
-    runs->lo[s] = lo;
-    runs->pre[s + 1] = lower_bound_idx(g, n, c1) - lo;
+    runs->lo[threadIdx.x] = lo;
+    runs->pre[threadIdx.x + 1] = lower_bound_idx(g, n, c1) - lo;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -162,9 +169,10 @@ __global__ void __launch_bounds__(kPermThreads, 1) permute_cols_kernel(float* __
   find_runs(m, S, c0, c1, &runs);      // contains the barriers that publish the mbarrier init
   const int total = runs.pre[S];
   for (int e = threadIdx.x; e < total; e += kPermThreads) {
-    int s = 0;
-    while (e >= runs.pre[s + 1]) ++s;
-    const int j = runs.lo[s] + (e - runs.pre[s]);
+    int i = 0;
+    while (e >= runs.pre[i + 1]) ++i;
+    const int s = m.s_first + i;
+    const int j = runs.lo[i] + (e - runs.pre[i]);
     map_col[e] = (uint16_t)(m.col_idx[m.col_off[s] + j] - c0);
     map_off[e] = (long long)s * m.rows_pad * m.ld + j;
   }
@@ -211,7 +219,7 @@ __global__ void __launch_bounds__(kPermThreads, 1) permute_cols_kernel(float* __
         }
       }
       if (blockIdx.x == 0) {   // pad columns [|G^s|, ld) of these rows are zero
-        for (int s = 0; s < S; ++s) {
+        for (int s = m.s_first; s < m.s_first + S; ++s) {
           const int cnt = m.col_off[s + 1] - m.col_off[s];
           const int npad = (int)m.ld - cnt;
           for (int e = threadIdx.x; e < npad * nrows; e += kPermThreads) {
@@ -256,13 +264,13 @@ template <bool GATHER>
 bool launch_permute_cols(const Launch& L, float* W, const SliceMap& m, int S, float* master, bf16* opw,
                          DeviceStatus* st) {
   constexpr int smem = 2 * kStageRows * kStageCols * (int)sizeof(float) + kStageCols * 8 + kStageCols * 2;
+  static std::once_flag once;     // one instance per direction; any host thread may come first
   static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(permute_cols_kernel<GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-        cudaSuccess)
-      return false;
-    configured = true;
-  }
+  std::call_once(once, [] {
+    configured = cudaFuncSetAttribute(permute_cols_kernel<GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      smem) == cudaSuccess;
+  });
+  if (!configured) return false;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int64_t chunks = ceil_div(m.full_cols, kStageCols), blocks = ceil_div(m.full_rows, kStageRows);
@@ -299,7 +307,7 @@ __global__ void copy_out_kernel(const float* __restrict__ packed, int64_t ld, in
 void gather_slices(const Launch& L, const float* W, const SliceMap& m, int S, float* master,
                    bf16* opw, DeviceStatus* st) {
   if (staged_ok(m, S) && launch_permute_cols<true>(L, const_cast<float*>(W), m, S, master, opw, st)) return;
-  dim3 grid((unsigned)ceil_div(m.ld, kThreads), (unsigned)ceil_div(m.rows_pad, kRowsPerCta), S);
+  dim3 grid((unsigned)ceil_div(m.ld, kThreads), (unsigned)std::min<int64_t>(ceil_div(m.rows_pad, kRowsPerCta), 65535), S);
   gather_kernel<<<grid, kThreads, 0, L.stream>>>(W, m, master, opw);
   L.count();
 }
@@ -307,7 +315,7 @@ void gather_slices(const Launch& L, const float* W, const SliceMap& m, int S, fl
 void scatter_slices(const Launch& L, float* W, const SliceMap& m, int S, const float* master,
                     DeviceStatus* st) {
   if (staged_ok(m, S) && launch_permute_cols<false>(L, W, m, S, const_cast<float*>(master), nullptr, st)) return;
-  dim3 grid((unsigned)ceil_div(m.ld, kThreads), (unsigned)ceil_div(m.rows_pad, kRowsPerCta), S);
+  dim3 grid((unsigned)ceil_div(m.ld, kThreads), (unsigned)std::min<int64_t>(ceil_div(m.rows_pad, kRowsPerCta), 65535), S);
   scatter_kernel<<<grid, kThreads, 0, L.stream>>>(W, m, master);
   L.count();
 }

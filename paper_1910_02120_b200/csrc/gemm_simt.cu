@@ -50,8 +50,11 @@ __global__ void __launch_bounds__(kThreads) gemm_simt_kernel(GemmArgs<T> a) {
   constexpr int TM = BM / 16, TN = BN / 16;      // outputs per thread
   __shared__ float As[BK][BM + 1];
   __shared__ float Bs[BK][BN + 1];
+  // blockIdx.x runs over (m tile, n tile) pairs, n fastest: the x dimension of a grid has room
+  // for 2^31 - 1 blocks, the y dimension only for 65535
   const int g = blockIdx.z;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int n_tiles = (a.N + BN - 1) / BN;
+  const int m0 = (int)(blockIdx.x / n_tiles) * BM, n0 = (int)(blockIdx.x % n_tiles) * BN;
   const int tid = threadIdx.x;
   const int ty = tid / 16, tx = tid % 16;
   const T* A = a.A + (int64_t)g * a.a_sg;
@@ -133,10 +136,10 @@ void gemm_simt(const Launch& L, const GemmArgs<T>& a) {
   // few large tiles leave most of the 148 SMs idle: use 32x32 tiles until every SM has two
   const int64_t big = ceil_div(a.N, 64) * ceil_div(a.M, 64) * a.G;
   if (big >= 296) {
-    dim3 grid((unsigned)ceil_div(a.N, 64), (unsigned)ceil_div(a.M, 64), (unsigned)a.G);
+    dim3 grid((unsigned)(ceil_div(a.N, 64) * ceil_div(a.M, 64)), 1, (unsigned)a.G);
     gemm_simt_kernel<T, 64, 64><<<grid, kThreads, 0, L.stream>>>(a);
   } else {
-    dim3 grid((unsigned)ceil_div(a.N, 32), (unsigned)ceil_div(a.M, 32), (unsigned)a.G);
+    dim3 grid((unsigned)(ceil_div(a.N, 32) * ceil_div(a.M, 32)), 1, (unsigned)a.G);
     gemm_simt_kernel<T, 32, 32><<<grid, kThreads, 0, L.stream>>>(a);
   }
   L.count();

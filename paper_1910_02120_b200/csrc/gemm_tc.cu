@@ -782,12 +782,13 @@ EncodeTiledFn encode_fn() {
 
 int sm_count() {
   static int n = 0;
-  if (n == 0) {
+  static std::once_flag once;
+  std::call_once(once, [] {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
       n = 148;
-  }
+  });
   return n;
 }
 

@@ -154,7 +154,8 @@ ist_status fail(ist_ctx* c, ist_status code, const char* fmt, ...) {
 bool valid_shape(const int64_t* dims, int n_dims, int S, int precision, int max_batch, std::string* why) {
   if (!dims || n_dims < 2 || n_dims > 64) { *why = "layer_dims must hold 2..64 entries"; return false; }
   if (precision != IST_FP32 && precision != IST_BF16) { *why = "precision must be IST_FP32 or IST_BF16"; return false; }
-  if (max_batch < 1 || max_batch > (1 << 20)) { *why = "max_batch must be in 1..2^20"; return false; }
+  // a minibatch runs along the y dimension of several launch grids, which holds 65535 blocks
+  if (max_batch < 1 || max_batch > 65535) { *why = "max_batch must be in 1..65535"; return false; }
   if (S < 1) { *why = "S must be >= 1"; return false; }
   for (int i = 0; i < n_dims; ++i)
     if (dims[i] < 1 || dims[i] > (int64_t)1 << 30) { *why = "every layer width must be in 1..2^30"; return false; }
@@ -179,8 +180,15 @@ bool wide_head(const ist_ctx* c) { return c->precision == IST_BF16 && c->ld[c->t
 
 // delta_{l-1} = delta_l * W_l^T contracts over the width of layer l.  When that width is huge
 // (hundreds of thousands of classes) and the output small, the product has too few tiles to
-// fill the machine, so the contraction is cut into slices that run as separate tiles.
-int wanted_k_splits(int64_t K) { return K >= 16384 ? (int)std::min<int64_t>(64, ceil_div(K, 8192)) : 1; }
+// fill the machine, so the contraction is cut into slices that run as separate tiles.  A product
+// that already has a 256 x 256 tile for every pair of SMs is left whole: slices would only add
+// fp32 partial slabs to write and read back.
+int wanted_k_splits(int64_t K, int64_t out_cols, int S, int B) {
+  if (K < 16384) return 1;
+  const int64_t tiles = ceil_div(B, 256) * ceil_div(out_cols, 256) * S;
+  if (tiles >= 74) return 1;
+  return (int)std::min<int64_t>(64, ceil_div(K, 8192));
+}
 
 void make_plan(ist_ctx* c) {
   Plan& p = c->plan;
@@ -221,8 +229,10 @@ void make_plan(ist_ctx* c) {
   // fp32 partial products of k-split delta GEMMs (very wide layers only)
   size_t sk = 0;
   if (c->precision == IST_BF16)
-    for (int l = 2; l <= t; ++l)
-      sk = std::max(sk, (size_t)(wanted_k_splits(c->np[l]) > 1 ? wanted_k_splits(c->np[l]) : 0) * S * Bm * c->ld[l - 1] * 4);
+    for (int l = 2; l <= t; ++l) {   // batch 1 has the fewest tiles, hence the most slices any batch can ask for
+      const int ks = wanted_k_splits(c->np[l], c->np[l - 1], S, 1);
+      sk = std::max(sk, (size_t)(ks > 1 ? ks : 0) * S * Bm * c->ld[l - 1] * 4);
+    }
   p.splitk = p.take(sk);
 }
 
@@ -291,8 +301,9 @@ uint64_t splitmix64_next(uint64_t* state) {
 }
 
 // Slice map of layer l (1..t): rows follow hidden layer l-1's partition, columns layer l's.
-SliceMap slice_map(const ist_ctx* c, int l) {
+SliceMap slice_map(const ist_ctx* c, int l, int s_first = 0) {
   SliceMap m{};
+  m.s_first = s_first;
   const bool rows_indexed = l > 1, cols_indexed = l < c->t;
   m.row_idx = rows_indexed ? c->idx(l - 1) : nullptr;
   m.row_off = rows_indexed ? c->off(l - 1) : nullptr;
@@ -305,8 +316,9 @@ SliceMap slice_map(const ist_ctx* c, int l) {
   return m;
 }
 
-SliceMap bias_map(const ist_ctx* c, int l) {
+SliceMap bias_map(const ist_ctx* c, int l, int s_first = 0) {
   SliceMap m{};
+  m.s_first = s_first;
   const bool cols_indexed = l < c->t;
   m.col_idx = cols_indexed ? c->idx(l) : nullptr;
   m.col_off = cols_indexed ? c->off(l) : nullptr;
@@ -538,7 +550,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.mask = act(l - 1); g.mask_ld = c->ld[l - 1]; g.mask_sg = Bm * c->ld[l - 1];
         g.out = delta(l - 1); g.out_ld = c->ld[l - 1]; g.out_sg = Bm * c->ld[l - 1];
         Scope sc(c, IST_K_DX);
-        const int want = bf ? wanted_k_splits(c->np[l]) : 1;
+        const int want = bf ? wanted_k_splits(c->np[l], c->np[l - 1], S, B) : 1;
         if (want > 1) {
           if (!split_delta_gemm(c, g, want, B))
             return fail(c, IST_ERR_UNSUPPORTED, "k-split delta GEMM of layer %d cannot be launched", l);
@@ -697,10 +709,11 @@ extern "C" ist_status ist_partition(ist_ctx* c, uint64_t seed) {
                         : partition_layer(L, layer_seed, (int)c->N[l], S, ps, c->idx(l), c->off(l), c->status());
     if (!ok) return fail(c, IST_ERR_UNSUPPORTED, "S = %d exceeds what the partition kernels support (768)", S);
   }
+  // only the subnets this context trains are gathered (Sec. 2.3: a site receives its own slices)
   for (int l = 1; l <= t; ++l) {
     Scope sc(c, IST_K_GATHER);
-    gather_slices(L, c->W[l - 1], slice_map(c, l), S, c->master(l), c->opw(l), c->status());
-    gather_slices(L, c->b[l - 1], bias_map(c, l), S, c->bias(l), nullptr, c->status());
+    gather_slices(L, c->W[l - 1], slice_map(c, l, c->sub_first), c->sub_count, c->master(l), c->opw(l), c->status());
+    gather_slices(L, c->b[l - 1], bias_map(c, l, c->sub_first), c->sub_count, c->bias(l), nullptr, c->status());
   }
   IST_CUDA(c, cudaGetLastError());
   c->state = ST_PARTITIONED;
@@ -721,16 +734,31 @@ extern "C" ist_status ist_get_partition(ist_ctx* c, int hidden_layer, int32_t* i
   return IST_OK;
 }
 
+namespace {
+// |G_l^s| under the partition in place; the input and output layers belong to every subnet whole
+int64_t group_size(const ist_ctx* c, int l, int s) {
+  if (l == 0 || l == c->t) return c->N[l];
+  if (c->rule == IST_PART_IID) return c->group_count[l][s];
+  return c->N[l] / c->S + (s < c->N[l] % c->S ? 1 : 0);
+}
+}  // namespace
+
+extern "C" ist_status ist_subnet_slice_shape(ist_ctx* c, int layer, int s, int64_t* rows_out_host,
+                                             int64_t* cols_out_host) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state != ST_PARTITIONED) return fail(c, IST_ERR_STATE, "no partition in place");
+  if (layer < 1 || layer > c->t || s < 0 || s >= c->S) return fail(c, IST_ERR_ARG, "layer or subnet out of range");
+  if (rows_out_host) *rows_out_host = group_size(c, layer - 1, s);
+  if (cols_out_host) *cols_out_host = group_size(c, layer, s);
+  return IST_OK;
+}
+
 extern "C" ist_status ist_get_subnet_params(ist_ctx* c, int layer, int s, float* W_out_dev,
                                             float* b_out_dev) {
   if (!c) return IST_ERR_ARG;
   if (c->state != ST_PARTITIONED) return fail(c, IST_ERR_STATE, "no partition in place");
   if (layer < 1 || layer > c->t || s < 0 || s >= c->S) return fail(c, IST_ERR_ARG, "layer or subnet out of range");
-  auto count = [&](int l) -> int64_t {   // |G_l^s| (balanced split), full width at the ends
-    if (l == 0 || l == c->t) return c->N[l];
-    if (c->rule == IST_PART_IID) return c->group_count[l][s];
-    return c->N[l] / c->S + (s < c->N[l] % c->S ? 1 : 0);
-  };
+  auto count = [&](int l) { return group_size(c, l, s); };
   Launch L = c->launch();
   if (W_out_dev)
     copy_out_slice(L, c->master(layer) + (int64_t)s * c->slice_elems(layer), c->ld[layer],

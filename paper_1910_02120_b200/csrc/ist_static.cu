@@ -33,7 +33,15 @@ static __device__ __align__(256) unsigned char g_scratch[kStaticScratchBytes];
 std::mutex g_mutex;
 void* g_scratch_addr[kMaxDevices] = {};
 
-// Device address of g_scratch on the current device (looked up once per device).
+// Device address of g_scratch on the current device (looked up once per device), or null if no
+// call has looked it up yet.
+void* scratch_address_if_known() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lk(g_mutex);
+  return g_scratch_addr[dev];
+}
+
 ist_status scratch_address(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return IST_ERR_CUDA;
@@ -86,4 +94,15 @@ extern "C" ist_status ist_partition_layer_static(uint64_t seed, int hidden_layer
   if (!partition_layer(L, layer_seed, N, S, sc, idx_out_dev, off_out_dev, reinterpret_cast<DeviceStatus*>(base)))
     return IST_ERR_UNSUPPORTED;
   return cudaGetLastError() == cudaSuccess ? IST_OK : IST_ERR_CUDA;
+}
+
+
+extern "C" ist_status ist_static_partition_status(void* cuda_stream) {
+  void* base = scratch_address_if_known();
+  if (!base) return IST_OK;   // the entry point has not run on this device: nothing to report
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  DeviceStatus h{};
+  if (cudaMemcpyAsync(&h, base, sizeof h, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return IST_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return IST_ERR_CUDA;
+  return h.code == 0 ? IST_OK : (ist_status)h.code;
 }

@@ -47,7 +47,9 @@ struct SliceMap {
   const int32_t* col_off;
   int64_t full_rows, full_cols;  // N_{l-1}, N_l (row stride of the full matrix = full_cols)
   int64_t rows_pad, ld;          // packed slice: [S][rows_pad][ld]
+  int s_first;                   // first subnet a launch covers (it covers S consecutive ones)
 };
+// S = number of subnets moved, starting at m.s_first; master / opw point at subnet 0's slab.
 void gather_slices(const Launch& L, const float* W, const SliceMap& m, int S, float* master,
                    bf16* opw, DeviceStatus* st);
 void scatter_slices(const Launch& L, float* W, const SliceMap& m, int S, const float* master,

@@ -61,6 +61,14 @@ def test_create_rejects_bad_workspace_without_a_device(api):
     assert api.lib.ist_partition(None, 1) == api.IST_ERR_ARG
 
 
+def test_slice_shape_and_static_status_need_no_device_to_refuse(api):
+    r, c = ctypes.c_int64(-1), ctypes.c_int64(-1)
+    assert api.lib.ist_subnet_slice_shape(None, 1, 0, ctypes.byref(r), ctypes.byref(c)) == api.IST_ERR_ARG
+    assert (r.value, c.value) == (-1, -1)
+    assert api.ist_workspace_bytes([8, 4, 3], 2, api.IST_FP32, 65536) == 0           # batch beyond a launch grid's rows
+    assert api.ist_workspace_bytes([8, 4, 3], 2, api.IST_FP32, 65535) > 0
+
+
 def test_normalisation_entry_points_reject_null_contexts(api):
     assert api.lib.ist_norm_workspace_bytes(None) == 0
     assert api.lib.ist_enable_normalization(None, ctypes.c_float(1e-5), None, 0) == api.IST_ERR_ARG

@@ -52,6 +52,25 @@ def test_static_partition_matches_the_workspace_path_twice_in_a_row():
     assert np.array_equal(idx2.cpu().numpy(), _reference_partition(api, [8, 4096, 5], 8, 123)[0][0])
 
 
+def test_static_partition_takes_no_device_memory_and_reports_its_status():
+    """The point of the entry point: free device memory is the same before and after warmed-up calls
+    (the first call's symbol look-up is done by then), and the kernels' bounds-check word reads OK."""
+    import torch
+    from paper_1910_02120_b200 import api
+    N, S = 30000, 16
+    idx = torch.empty(N, dtype=torch.int32, device="cuda:0")
+    off = torch.empty(S + 1, dtype=torch.int32, device="cuda:0")
+    assert api.ist_partition_layer_static(5, 1, N, S, idx, off) == api.IST_OK      # warm-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for seed in range(6, 12):
+        assert api.ist_partition_layer_static(seed, 2, N, S, idx, off) == api.IST_OK
+    assert api.ist_static_partition_status() == api.IST_OK
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
+    assert np.array_equal(np.sort(idx.cpu().numpy()), np.arange(N))
+
+
 def test_static_partition_refuses_sizes_beyond_its_scratch():
     import torch
     from paper_1910_02120_b200 import api
