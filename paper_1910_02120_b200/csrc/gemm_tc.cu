@@ -35,6 +35,17 @@
 // memory tile is 128-byte swizzled in both cases and the UMMA descriptors say which.  Rows and
 // columns beyond the tensor extents are zero-filled by TMA loads and dropped by TMA stores.
 //
+// One launch may run several products of the same kind ("problems": the same operand layouts, tile
+// shape and epilogue, e.g. the weight updates of all layers of a step).  Their tiles form one flat
+// list that the CTAs walk in order, so that a small product costs a few tiles instead of a launch
+// and no SM idles between one product's last wave and the next one's first.  A problem may be
+// chained to the one before it in the list (its A operand is that problem's output, as in
+// a_l = relu(a_{l-1} W_l + b_l) or delta_{l-1} = (delta_l W_l^T) * mask): its tiles then wait
+// until the rows they read are complete, through one counter per (group, block of tile rows)
+// that the storing threads of the producer bump after their stores have completed.  Tiles are
+// claimed in list order by CTAs that are all resident at once, and a tile depends only on
+// earlier tiles, so the waits always end; they are bounded like every other wait here.
+//
 // Every wait is bounded: after about a second without progress a role records
 // IST_ERR_DEVICE_TIMEOUT in the status word, raises the CTA's abort flag and all roles fall
 // through to the common exit, where tensor memory is released.
@@ -223,21 +234,67 @@ __host__ __device__ constexpr uint32_t make_idesc(int a_mn, int b_mn, int n, int
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-struct TcArgs {
+constexpr int kMaxProblems = 4;
+
+// One product of a launch.  Tiles tile_end(previous) .. tile_end - 1 of the flat list are its.
+struct TcProblem {
   int M, N, K;            // M, N: bounds of the output rows / columns the epilogue touches
   int m_tiles, n_tiles, G;
   int k_splits, kb_per_split;   // the k range may be cut into slices that run as separate tiles
   int a_gmul, b_gmul;     // 1 if the operand has one slab per group, 0 if all groups share it
+  int tile_end;
   const float* bias; long long bias_sg;
+  // chaining: counters [G][m_tiles]; a tile of (g, mt) may load A once wait_ctr[g * m_tiles + mt]
+  // has reached wait_target; a storer adds the chunks it has stored for (g, mt) to signal_ctr
+  const unsigned* wait_ctr; unsigned wait_target;
+  unsigned* signal_ctr;
+};
+
+struct TcArgs {
+  int n_problems, total_tiles;
+  TcProblem p[kMaxProblems];
   float lr;
   DeviceStatus* status;
-  // wide softmax head (see GemmArgs)
+  // wide softmax head (see GemmArgs); single-problem launches only
   float2* lse_part;
   const float* lse; long long lse_sg;
   const int32_t* labels; long long labels_sg;
   float* label_logit;
   float inv_rows;
 };
+
+struct TcMaps {
+  CUtensorMap a[kMaxProblems], b[kMaxProblems];
+  CUtensorMap c32[kMaxProblems];     // fp32 chunks: logits out, master in/out
+  CUtensorMap c16[kMaxProblems];     // bf16 chunks out: activations, delta, weights
+  CUtensorMap aux16[kMaxProblems];   // bf16 chunks in: ReLU mask
+};
+
+// Where a tile of the flat list lies: problem, tile row / column, output slab (group and k slice).
+struct TileAt {
+  int pi, mt, nt, slab;
+};
+__device__ __forceinline__ TileAt locate(const TcArgs& a, int tile, int& pi) {
+  while (tile >= a.p[pi].tile_end) ++pi;       // tiles are visited in increasing order
+  const TcProblem& pr = a.p[pi];
+  const int lt = tile - (pi ? a.p[pi - 1].tile_end : 0);
+  TileAt t;
+  t.pi = pi;
+  t.mt = lt % pr.m_tiles;
+  t.nt = (lt / pr.m_tiles) % pr.n_tiles;
+  t.slab = lt / (pr.m_tiles * pr.n_tiles);
+  return t;
+}
+
+__device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // Chunk staging: a ring of fp32 areas ([128][32] floats, 128-byte swizzle) and / or a ring of
 // bf16 areas ([128][32] bf16, 64-byte swizzle); kAux says whether chunks are loaded before use
@@ -283,11 +340,7 @@ __device__ __forceinline__ uint4* b16_unit(uint8_t* area, int r, int u) {
 
 template <int A_MN, int B_MN, int BN, int STAGES, int NS, int EPI, int PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmC32,   // fp32 chunks: logits out, master in/out
-               const __grid_constant__ CUtensorMap tmC16,   // bf16 chunks out: activations, delta, weights
-               const __grid_constant__ CUtensorMap tmAux16, // bf16 chunks in: ReLU mask
-               TcArgs a) {
+gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcArgs a) {
   using ET = EpiTraits<EPI>;
   constexpr int BNL = BN / PAIR;   // rows of the B tile this CTA loads
   constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BNL * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
@@ -309,17 +362,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int num_kb = (a.K + BK - 1) / BK;
-  const int total_tiles = a.m_tiles * a.n_tiles * a.G * a.k_splits;   // tiles of (128 * PAIR) x BN x k slice
+  const int total_tiles = a.total_tiles;             // tiles of (128 * PAIR) x BN x k slice, all problems
   const int rank = PAIR == 2 ? (int)cluster_ctarank() : 0;
   const int unit = blockIdx.x / PAIR, n_units = gridDim.x / PAIR;   // a unit = a CTA or a pair
 
   if (threadIdx.x == 32) {   // the maps this instance copies through; they do not depend on the previous kernel
-    prefetch_map(&tmA);
-    prefetch_map(&tmB);
-    if (ET::k32) prefetch_map(&tmC32);
-    if (ET::k16) prefetch_map(&tmC16);
-    if (EPI == EPI_RELU_MASK) prefetch_map(&tmAux16);
+    for (int i = 0; i < a.n_problems; ++i) {
+      prefetch_map(&maps.a[i]);
+      prefetch_map(&maps.b[i]);
+      if (ET::k32) prefetch_map(&maps.c32[i]);
+      if (ET::k16) prefetch_map(&maps.c16[i]);
+      if (EPI == EPI_RELU_MASK) prefetch_map(&maps.aux16[i]);
+    }
   }
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -369,14 +423,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 0) {
     // ---------------------------------------------------------------- operand loads
     if (lane == 0) {
-      int it = 0;
+      int it = 0, pi = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
-        const int m0 = (tile % a.m_tiles) * (BM * PAIR) + rank * BM;     // this CTA's rows of A
-        const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN + rank * BNL;   // this CTA's rows of B
-        const int rest = tile / (a.m_tiles * a.n_tiles);
-        const int g = rest / a.k_splits;
-        const int kb0 = (rest % a.k_splits) * a.kb_per_split, kb1 = min(num_kb, kb0 + a.kb_per_split);
+        const TileAt at = locate(a, tile, pi);
+        const TcProblem& pr = a.p[pi];
+        const CUtensorMap* tmA = &maps.a[pi];
+        const CUtensorMap* tmB = &maps.b[pi];
+        const int m0 = at.mt * (BM * PAIR) + rank * BM;     // this CTA's rows of A
+        const int n0 = at.nt * BN + rank * BNL;             // this CTA's rows of B
+        const int g = at.slab / pr.k_splits;
+        const int num_kb = (pr.K + BK - 1) / BK;
+        const int kb0 = (at.slab % pr.k_splits) * pr.kb_per_split, kb1 = min(num_kb, kb0 + pr.kb_per_split);
+        const int ga = g * pr.a_gmul, gb = g * pr.b_gmul;
+        if (pr.wait_ctr) {
+          // A is the output of the problem before this one: wait until every chunk of these rows
+          // has been stored (the storers count them), then order the copies below after that
+          const unsigned* ctr = pr.wait_ctr + (long long)g * pr.m_tiles + at.mt;
+          const long long t0 = clock64();
+          while ((int)(ld_acquire(ctr) - pr.wait_target) < 0) {
+            if (*abortp) { ok = false; break; }
+            if (clock64() - t0 > kWaitLimitCycles) {
+              *abortp = 1;
+              report(a.status, -6, SITE_TC_PIPE, 8);
+              ok = false;
+              break;
+            }
+            __nanosleep(64);
+          }
+          if (!ok) break;
+          fence_proxy_async_all();
+        }
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           ok = mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abortp, a.status, 1);
@@ -390,32 +467,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (A_MN) {
 #pragma unroll
               for (int j = 0; j < BM / 64; ++j)
-                tma_load_3d_pair(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, kb * BK, g * a.a_gmul);
+                tma_load_3d_pair(sa + j * (BK * 128), tmA, bar, m0 + 64 * j, kb * BK, ga);
             } else {
-              tma_load_3d_pair(sa, &tmA, bar, kb * BK, m0, g * a.a_gmul);
+              tma_load_3d_pair(sa, tmA, bar, kb * BK, m0, ga);
             }
             if (B_MN) {
 #pragma unroll
               for (int j = 0; j < BNL / 64; ++j)
-                tma_load_3d_pair(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, kb * BK, g * a.b_gmul);
+                tma_load_3d_pair(sb + j * (BK * 128), tmB, bar, n0 + 64 * j, kb * BK, gb);
             } else {
-              tma_load_3d_pair(sb, &tmB, bar, kb * BK, n0, g * a.b_gmul);
+              tma_load_3d_pair(sb, tmB, bar, kb * BK, n0, gb);
             }
           } else {
             mbar_expect_tx(&full_bar[s], STAGE_BYTES);
             if (A_MN) {
 #pragma unroll
               for (int j = 0; j < BM / 64; ++j)
-                tma_load_3d(sa + j * (BK * 128), &tmA, &full_bar[s], m0 + 64 * j, kb * BK, g * a.a_gmul);
+                tma_load_3d(sa + j * (BK * 128), tmA, &full_bar[s], m0 + 64 * j, kb * BK, ga);
             } else {
-              tma_load_3d(sa, &tmA, &full_bar[s], kb * BK, m0, g * a.a_gmul);
+              tma_load_3d(sa, tmA, &full_bar[s], kb * BK, m0, ga);
             }
             if (B_MN) {
 #pragma unroll
               for (int j = 0; j < BNL / 64; ++j)
-                tma_load_3d(sb + j * (BK * 128), &tmB, &full_bar[s], n0 + 64 * j, kb * BK, g * a.b_gmul);
+                tma_load_3d(sb + j * (BK * 128), tmB, &full_bar[s], n0 + 64 * j, kb * BK, gb);
             } else {
-              tma_load_3d(sb, &tmB, &full_bar[s], kb * BK, n0, g * a.b_gmul);
+              tma_load_3d(sb, tmB, &full_bar[s], kb * BK, n0, gb);
             }
           }
         }
@@ -433,16 +510,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ---------------------------------------------------------------- MMA issue
     if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BN, BM * PAIR);
-      int it = 0, j = 0;
+      int it = 0, j = 0, pi = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
+        const TileAt at = locate(a, tile, pi);
+        const TcProblem& pr = a.p[pi];
         const int b = j & 1;
         ok = mbar_wait(&acc_empty[b], ((j >> 1) & 1) ^ 1, abortp, a.status, 2);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
-        const int kb0 = ((tile / (a.m_tiles * a.n_tiles)) % a.k_splits) * a.kb_per_split;
-        const int kb1 = min(num_kb, kb0 + a.kb_per_split);
+        const int num_kb = (pr.K + BK - 1) / BK;
+        const int kb0 = (at.slab % pr.k_splits) * pr.kb_per_split;
+        const int kb1 = min(num_kb, kb0 + pr.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           ok = mbar_wait(&full_bar[s], (it / STAGES) & 1, abortp, a.status, 3);
@@ -471,35 +551,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int q = warp & 3;                           // tensor-memory lane quarter of this warp
     const int wg = (warp - 2) >> 2;                   // this warp's group takes chunks with cq % 2 == wg
     const int r = q * 32 + lane;                      // row of the tile owned by this thread
-    int cq = 0, j = 0;
+    int cq = 0, j = 0, pi = 0, pi_next = 0;
     bool ok = true;
     // per-tile epilogue inputs, requested one tile ahead (see below)
     float next_bias[NCH];
     float next_lse = 0.f;
     int next_label = -1;
     auto prefetch_tile_inputs = [&](int tile) {
-      const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
-      const int g = tile / (a.m_tiles * a.n_tiles);
+      const TileAt at = locate(a, tile, pi_next);
+      const TcProblem& pr = a.p[pi_next];
+      const int n0 = at.nt * BN;
       if (EPI == EPI_BIAS_RELU || EPI == EPI_BIAS_F32 || EPI == EPI_LSE_PART || EPI == EPI_SOFTMAX_DELTA) {
-        const float* bias = a.bias ? a.bias + (long long)(g / a.k_splits) * a.bias_sg : nullptr;
+        const float* bias = pr.bias ? pr.bias + (long long)(at.slab / pr.k_splits) * pr.bias_sg : nullptr;
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           const int n = n0 + c * CH + lane;
-          next_bias[c] = (bias && n < a.N) ? __ldg(bias + n) : 0.f;
+          next_bias[c] = (bias && n < pr.N) ? __ldg(bias + n) : 0.f;
         }
       }
       if (EPI == EPI_SOFTMAX_DELTA) {
-        const int row = (tile % a.m_tiles) * (BM * PAIR) + rank * BM + r;
-        next_lse = row < a.M ? __ldg(a.lse + (long long)g * a.lse_sg + row) : 0.f;
-        next_label = row < a.M ? __ldg(a.labels + (long long)g * a.labels_sg + row) : -1;
+        const int row = at.mt * (BM * PAIR) + rank * BM + r;
+        next_lse = row < pr.M ? __ldg(a.lse + (long long)at.slab * a.lse_sg + row) : 0.f;
+        next_label = row < pr.M ? __ldg(a.labels + (long long)at.slab * a.labels_sg + row) : -1;
       }
     };
 #pragma unroll
     for (int c = 0; c < NCH; ++c) next_bias[c] = 0.f;
     if (unit < total_tiles) prefetch_tile_inputs(unit);
     for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
-      const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
-      const int g = tile / (a.m_tiles * a.n_tiles);   // output slab (group, k slice)
+      const TileAt at = locate(a, tile, pi);
+      const int pN = a.p[pi].N, pM = a.p[pi].M, p_ntiles = a.p[pi].n_tiles;
+      const int n0 = at.nt * BN;
+      const int g = at.slab;                          // output slab (group, k slice)
       const int b = j & 1;
       // Bias of the tile's columns: lane l keeps column 32 * c + l of every chunk c, and the chunk
       // code reads the 32 values of its chunk with warp shuffles.  The values (and the per-row
@@ -508,7 +591,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       float bias_reg[NCH];
 #pragma unroll
       for (int c = 0; c < NCH; ++c) bias_reg[c] = next_bias[c];
-      const int row = (tile % a.m_tiles) * (BM * PAIR) + rank * BM + r;   // this thread's row of the output
+      const int row = at.mt * (BM * PAIR) + rank * BM + r;   // this thread's row of the output
       float run_max = -INFINITY, run_sum = 0.f;       // EPI_LSE_PART: over this warp group's chunks
       const float row_lse = next_lse * kLog2e;        // log-sum-exp in the log2 domain
       const int row_label = next_label;
@@ -520,7 +603,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll 1
       for (int c = 0; c < NCH; ++c, ++cq) {
         const int nc = n0 + c * CH;
-        if (nc >= a.N) break;                         // CTA-uniform
+        if (nc >= pN) break;                          // CTA-uniform
         // A slot always belongs to the same warp group, so that the group sees the slot's barrier
         // phases in order (a parity wait cannot tell phase p from phase p + 2); every configuration
         // that stores through the ring has an even number of slots, so the groups alternate.
@@ -581,10 +664,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             z[e] = fmaf(__uint_as_float(acc[e]), kLog2e, __shfl_sync(0xffffffffu, bl, e));
           if (EPI == EPI_LSE_PART) {
             // running (max, sum of 2^(z - max)) of this row over the chunks this warp group sees
-            if (nc + CH > a.N) {                         // CTA-uniform: the last, ragged chunk
+            if (nc + CH > pN) {                          // CTA-uniform: the last, ragged chunk
 #pragma unroll
               for (int e = 0; e < 32; ++e)
-                if (nc + e >= a.N) z[e] = -INFINITY;     // pad columns do not count
+                if (nc + e >= pN) z[e] = -INFINITY;      // pad columns do not count
             }
             // four independent chains each, so that the maxima, the ex2 and the sums overlap
             float m4[4] = {z[0], z[1], z[2], z[3]};
@@ -604,19 +687,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               for (int e = 0; e < 8; ++e) o[e] = ex2_approx(z[8 * u + e] - row_lse) * a.inv_rows;
               *b16_unit(b16, r, u) = pack8(o);
             }
-            if (nc + CH > a.N) {                         // zero the pad columns of the ragged chunk
+            if (nc + CH > pN) {                          // zero the pad columns of the ragged chunk
 #pragma unroll
               for (int e = 0; e < 32; ++e)
-                if (nc + e >= a.N)
+                if (nc + e >= pN)
                   reinterpret_cast<bf16*>(b16_unit(b16, r, e >> 3))[e & 7] = __float2bfloat16_rn(0.f);
             }
-            const int at = row_label - nc;               // the label's column, if it is in this chunk
-            if (at >= 0 && at < CH && row < a.M) {
+            const int lat = row_label - nc;              // the label's column, if it is in this chunk
+            if (lat >= 0 && lat < CH && row < pM) {
               float zl = 0.f;
 #pragma unroll
               for (int e = 0; e < 32; ++e)
-                if (e == at) zl = z[e];
-              reinterpret_cast<bf16*>(b16_unit(b16, r, at >> 3))[at & 7] =
+                if (e == lat) zl = z[e];
+              reinterpret_cast<bf16*>(b16_unit(b16, r, lat >> 3))[lat & 7] =
                   __float2bfloat16_rn((ex2_approx(zl - row_lse) - 1.f) * a.inv_rows);
               a.label_logit[(long long)g * a.lse_sg + row] = zl * 0.6931471805599453f;
             }
@@ -649,10 +732,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
       if (!ok) break;
-      if (EPI == EPI_LSE_PART && row < a.M) {
+      if (EPI == EPI_LSE_PART && row < pM) {
         // two partials per tile (one per warp group), combined by lse_combine
-        const int tn = (tile / a.m_tiles) % a.n_tiles;
-        a.lse_part[((long long)g * (2 * a.n_tiles) + 2 * tn + wg) * a.M + row] = make_float2(run_max, run_sum);
+        a.lse_part[((long long)g * (2 * p_ntiles) + 2 * at.nt + wg) * pM + row] = make_float2(run_max, run_sum);
       }
       tc_fence_before();
       __syncwarp();
@@ -663,21 +745,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == kAuxWarp) {
     // ---------------------------------------------------------------- epilogue input loads
     if (ET::kAux && lane == 0) {
-      int cq = 0;
+      int cq = 0, pi = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
-        const int m0 = (tile % a.m_tiles) * (BM * PAIR) + rank * BM;
-        const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
-        const int g = tile / (a.m_tiles * a.n_tiles);
+        const TileAt at = locate(a, tile, pi);
+        const int pN = a.p[pi].N;
+        const int m0 = at.mt * (BM * PAIR) + rank * BM;
+        const int n0 = at.nt * BN;
+        const int g = at.slab;
         for (int c = 0; c < NCH; ++c, ++cq) {
           const int nc = n0 + c * CH;
-          if (nc >= a.N) break;
+          if (nc >= pN) break;
           const int slot = cq % NS;
           ok = mbar_wait(&slot_empty[slot], ((cq / NS) & 1) ^ 1, abortp, a.status, 6);
           if (!ok) break;
           mbar_expect_tx(&slot_full[slot], AUX_BYTES);
-          if (EPI == EPI_SGD) tma_load_3d(slots + slot * SLOT_BYTES, &tmC32, &slot_full[slot], nc, m0, g);
-          else tma_load_3d(slots + slot * SLOT_BYTES + F32_BYTES, &tmAux16, &slot_full[slot], nc, m0, g);
+          if (EPI == EPI_SGD) tma_load_3d(slots + slot * SLOT_BYTES, &maps.c32[pi], &slot_full[slot], nc, m0, g);
+          else tma_load_3d(slots + slot * SLOT_BYTES + F32_BYTES, &maps.aux16[pi], &slot_full[slot], nc, m0, g);
         }
       }
       if (!ok) {
@@ -691,15 +775,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ---------------------------------------------------------------- chunk stores
     if (kStore && lane == 0) {
       const int sj = warp - kStoreWarp0;
-      int cq = 0;
+      int cq = 0, pi = 0, pi_next = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
-        const int m0 = (tile % a.m_tiles) * (BM * PAIR) + rank * BM;
-        const int n0 = ((tile / a.m_tiles) % a.n_tiles) * BN;
-        const int g = tile / (a.m_tiles * a.n_tiles);
+        const TileAt at = locate(a, tile, pi);
+        const TcProblem& pr = a.p[pi];
+        const int m0 = at.mt * (BM * PAIR) + rank * BM;
+        const int n0 = at.nt * BN;
+        const int g = at.slab;
+        unsigned stored = 0;                 // chunks of this tile this thread has stored
         for (int c = 0; c < NCH; ++c, ++cq) {
           const int nc = n0 + c * CH;
-          if (nc >= a.N) break;
+          if (nc >= pr.N) break;
           const int slot = cq % NS;
           // a slot always belongs to the same storer, so that storer sees the slot's barrier
           // phases in order (a parity wait cannot tell phase p from phase p + 2)
@@ -707,9 +794,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           ok = mbar_wait(&chunk_done[slot], (cq / NS) & 1, abortp, a.status, 7);
           if (!ok) break;
           uint8_t* f32 = slots + slot * SLOT_BYTES;
-          if (ET::k32) tma_store_3d(&tmC32, f32, nc, m0, g);
-          if (ET::k16) tma_store_3d(&tmC16, f32 + F32_BYTES, nc, m0, g);
+          if (ET::k32) tma_store_3d(&maps.c32[pi], f32, nc, m0, g);
+          if (ET::k16) tma_store_3d(&maps.c16[pi], f32 + F32_BYTES, nc, m0, g);
           tma_commit_group();
+          ++stored;
           if (EPI == EPI_SGD && PAIR == 2) {
             // The same chunk of this unit's next tile is asked into L2 now, one tile ahead of its
             // load, so that the load finds it there.  The request is issued here, where the
@@ -718,15 +806,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // high) the requests measured slower than going without.
             const int nt = tile + n_units;
             if (nt < total_tiles) {
-              const int pn = ((nt / a.m_tiles) % a.n_tiles) * BN + c * CH;
-              if (pn < a.N)
-                tma_prefetch_l2_3d(&tmC32, pn, (nt % a.m_tiles) * (BM * PAIR) + rank * BM, nt / (a.m_tiles * a.n_tiles));
+              const TileAt nx = locate(a, nt, pi_next);
+              const int pn = nx.nt * BN + c * CH;
+              if (pn < a.p[pi_next].N)
+                tma_prefetch_l2_3d(&maps.c32[pi_next], pn, nx.mt * (BM * PAIR) + rank * BM, nx.slab);
             }
           }
           // once the store has read the slot it can be refilled (by the loader) or rewritten (by
           // the epilogue warps); the write to global memory completes in the background
           tma_wait_read<0>();
           mbar_arrive(&slot_empty[slot]);
+        }
+        if (ok && pr.signal_ctr && stored) {
+          // a later problem of this launch reads these rows: once this thread's stores of the tile
+          // have completed, add them to the row block's count (release: the reader acquires it)
+          tma_wait_all();
+          fence_proxy_async_all();
+          red_release_add(pr.signal_ctr + (long long)(g / pr.k_splits) * pr.m_tiles + at.mt, stored);
         }
       }
       tma_wait_all();                // all stores complete before the CTA exits
@@ -838,20 +934,19 @@ bool make_map(CUtensorMap* out, const void* base, int elem_bytes, long long inne
   return true;
 }
 
-struct Maps {
-  CUtensorMap a, b, c32, c16, aux16;
-};
-
 template <int A_MN, int B_MN, int BN, int STAGES, int NS, int EPI, int PAIR>
-bool launch(const Launch& L, const Maps& m, const TcArgs& t) {
+bool launch(const Launch& L, const TcMaps& m, const TcArgs& t) {
   using ET = EpiTraits<EPI>;
   constexpr int slot_bytes = (ET::k32 ? BM * CH * 4 : 0) + (ET::k16 ? BM * CH * 2 : 0);
   constexpr int smem = STAGES * (BM * BK * 2 + (BN / PAIR) * BK * 2) + NS * slot_bytes + 1024;
   static_assert(smem <= 227 * 1024 - 512, "shared memory budget exceeded");
   auto kern = gemm_tc_kernel<A_MN, B_MN, BN, STAGES, NS, EPI, PAIR>;
-  static int max_units = 0;   // CTAs (PAIR = 1) or clusters (PAIR = 2) that can be resident at once
-  if (max_units == 0) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+  // CTAs (PAIR = 1) or clusters (PAIR = 2) that can be resident at once; looked up by whichever
+  // host thread launches this instance first
+  static int max_units = 0;
+  static std::once_flag once;
+  std::call_once(once, [&] {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return;
     if (PAIR == 2) {
       cudaLaunchConfig_t probe{};
       probe.gridDim = dim3(2 * (sm_count() / 2));
@@ -863,13 +958,14 @@ bool launch(const Launch& L, const Maps& m, const TcArgs& t) {
       probe.attrs = &attr;
       probe.numAttrs = 1;
       int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, kern, &probe) != cudaSuccess || n <= 0) return false;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &probe) != cudaSuccess || n <= 0) return;
       max_units = n < sm_count() / 2 ? n : sm_count() / 2;
     } else {
       max_units = sm_count();
     }
-  }
-  const int total = t.m_tiles * t.n_tiles * t.G * t.k_splits;
+  });
+  if (max_units <= 0) return false;
+  const int total = t.total_tiles;
   const int units = total < max_units ? total : max_units;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(PAIR * units);
@@ -889,7 +985,7 @@ bool launch(const Launch& L, const Maps& m, const TcArgs& t) {
   }
   cfg.attrs = attrs;
   cfg.numAttrs = n_attrs;
-  if (cudaLaunchKernelEx(&cfg, kern, m.a, m.b, m.c32, m.c16, m.aux16, t) != cudaSuccess) return false;
+  if (cudaLaunchKernelEx(&cfg, kern, m, t) != cudaSuccess) return false;
   L.count();
   return true;
 }
@@ -905,15 +1001,29 @@ bool gemm_tc_wait_selftest(const Launch& L, DeviceStatus* st, long long limit_cy
 // Tile shape.  Pairs of CTAs (256 x 256 tiles) are used when the problem has enough of them to
 // give every SM pair work; otherwise single CTAs with the widest of 256 / 128 / 64 columns that
 // still gives every SM a tile.  The weight-update epilogue keeps a chunk ring in shared memory
-// and stays at 128 columns when it runs on single CTAs.
+// and stays at 128 columns when it runs on single CTAs.  A batch of problems is judged by the
+// tiles of all of them together and must have one problem that qualifies for pairs by itself
+// (more than 128 rows and columns); the small ones then ride along on the same shape.
 struct TileChoice { int bn, pair; };
-TileChoice pick_tile(int M, int N, int G, int epi) {
+TileChoice pick_tile(const GemmArgs<bf16>* a, int n, int epi) {
   const int sms = sm_count();
-  auto tiles = [&](int bm, int bn) { return ceil_div(M, bm) * ceil_div(N, bn) * G; };
-  if (M > BM && N > 128 && 4 * tiles(2 * BM, 256) >= 3 * (sms / 2)) return {256, 2};
-  if (epi == EPI_SGD) return {(N > 64 && tiles(BM, 128) >= sms) ? 128 : 64, 1};
-  if (N > 128 && tiles(BM, 256) >= sms) return {256, 1};
-  if (N > 64 && tiles(BM, 128) >= sms) return {128, 1};
+  auto n_store = [&](int i) { return a[i].N_store > 0 ? a[i].N_store : a[i].N; };
+  auto tiles = [&](int bm, int bn) {
+    int64_t s = 0;
+    for (int i = 0; i < n; ++i)
+      s += ceil_div(a[i].M, bm) * ceil_div(n_store(i), bn) * a[i].G * (a[i].k_splits > 1 ? a[i].k_splits : 1);
+    return s;
+  };
+  bool pair_ok = false, wide = false, mid = false;
+  for (int i = 0; i < n; ++i) {
+    pair_ok |= a[i].M > BM && n_store(i) > 128;
+    wide |= n_store(i) > 128;
+    mid |= n_store(i) > 64;
+  }
+  if (pair_ok && 4 * tiles(2 * BM, 256) >= 3 * (sms / 2)) return {256, 2};
+  if (epi == EPI_SGD) return {(mid && tiles(BM, 128) >= sms) ? 128 : 64, 1};
+  if (wide && tiles(BM, 256) >= sms) return {256, 1};
+  if (mid && tiles(BM, 128) >= sms) return {128, 1};
   return {64, 1};
 }
 
@@ -928,62 +1038,132 @@ int gemm_tc_splits(int K, int want) {
   return (int)ceil_div(nkb, ceil_div(nkb, want));
 }
 
-bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
-  const int n_store = a.N_store > 0 ? a.N_store : a.N;
-  const bool a_mn = a.a_sm == 1 && a.a_sk != 1, b_mn = a.b_sn == 1 && a.b_sk != 1;
-  if (!a_mn && a.a_sk != 1) return false;
-  if (!b_mn && a.b_sk != 1) return false;
-  TileChoice tc = pick_tile(a.M, n_store, a.G * (a.k_splits > 1 ? a.k_splits : 1), a.epi);
-  if (a.epi == EPI_LSE_PART || a.epi == EPI_SOFTMAX_DELTA)   // the partials are laid out per 256-column tile
-    tc = TileChoice{256, a.M > BM ? 2 : 1};
-  const int bn = tc.bn, pair = tc.pair;
-  TcArgs t{};
-  t.M = a.M; t.N = n_store; t.K = a.K;
-  t.m_tiles = (int)ceil_div(a.M, BM * pair);
-  t.n_tiles = (int)ceil_div(n_store, bn);
-  t.G = a.G;
-  t.k_splits = 1;
-  t.kb_per_split = (int)ceil_div(a.K, BK);
-  if (a.k_splits > 1) {
-    if (a.epi != EPI_BIAS_F32 || a.bias) return false;   // slices are plain fp32 partial products
-    t.kb_per_split = (int)ceil_div(ceil_div(a.K, BK), a.k_splits);
-    t.k_splits = (int)ceil_div(ceil_div(a.K, BK), t.kb_per_split);
-    if (t.k_splits != a.k_splits) return false;           // caller sizes its buffer with gemm_tc_splits()
-  }
-  t.a_gmul = (a.G > 1 && a.a_sg != 0) ? 1 : 0;
-  t.b_gmul = (a.G > 1 && a.b_sg != 0) ? 1 : 0;
-  t.bias = a.bias; t.bias_sg = a.bias_sg;
-  t.lr = a.lr;
-  t.status = st;
-  t.lse_part = reinterpret_cast<float2*>(a.lse_part);
-  t.lse = a.lse; t.lse_sg = a.lse_sg;
-  t.labels = a.labels; t.labels_sg = a.labels_sg;
-  t.label_logit = a.label_logit;
-  t.inv_rows = a.inv_rows;
-  if ((long long)t.m_tiles * t.n_tiles * t.G > 0x7fffffffll) return false;
+int gemm_tc_max_batch() { return kMaxProblems; }
 
-  Maps m{};
-  // K-major operand: inner = K, outer = rows (M or N).  MN-major: inner = rows, outer = K.
-  const long long ga = t.a_gmul ? a.G : 1, gb = t.b_gmul ? a.G : 1;
-  const bool ok_a = a_mn ? make_map(&m.a, a.A, 2, a.M, a.K, ga, a.a_sk, a.a_sg, 64, BK, 128)
-                         : make_map(&m.a, a.A, 2, a.K, a.M, ga, a.a_sm, a.a_sg, 64, BM, 128);
-  const bool ok_b = b_mn ? make_map(&m.b, a.B, 2, a.N, a.K, gb, a.b_sk, a.b_sg, 64, BK, 128)
-                         : make_map(&m.b, a.B, 2, a.K, a.N, gb, a.b_sn, a.b_sg, 64, bn / pair, 128);
-  if (!ok_a || !ok_b) return false;
-  m.c32 = m.a; m.c16 = m.a; m.aux16 = m.a;   // placeholders for the maps an epilogue does not use
-  // Output / epilogue-input chunks: [G][M][n_store] row-major, boxes of 128 rows x 32 columns.
-  switch (a.epi) {
+// Counters a chain of n problems over G groups and up to max_rows output rows needs.
+size_t gemm_tc_chain_counters(int n, int G, int max_rows) { return (size_t)n * G * ceil_div(max_rows, BM); }
+
+bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmChain* chain, DeviceStatus* st) {
+  if (n < 1 || n > kMaxProblems) return false;
+  const GemmArgs<bf16>& a0 = ga[0];
+  const int epi = a0.epi;
+  const bool a_mn = a0.a_sm == 1 && a0.a_sk != 1, b_mn = a0.b_sn == 1 && a0.b_sk != 1;
+  for (int i = 0; i < n; ++i) {
+    const GemmArgs<bf16>& a = ga[i];
+    const bool ai = a.a_sm == 1 && a.a_sk != 1, bi = a.b_sn == 1 && a.b_sk != 1;
+    if (a.epi != epi || ai != a_mn || bi != b_mn) return false;     // one kernel instance serves the batch
+    if (!ai && a.a_sk != 1) return false;
+    if (!bi && a.b_sk != 1) return false;
+    if (n > 1 && a.k_splits > 1) return false;
+  }
+  if (n > 1 && epi != EPI_BIAS_RELU && epi != EPI_RELU_MASK && epi != EPI_SGD) return false;
+  if (chain && (epi == EPI_SGD || n < 2 || !chain->counters || !chain->totals)) return false;
+  TileChoice tc = pick_tile(ga, n, epi);
+  if (epi == EPI_LSE_PART || epi == EPI_SOFTMAX_DELTA)   // the partials are laid out per 256-column tile
+    tc = TileChoice{256, a0.M > BM ? 2 : 1};
+  const int bn = tc.bn, pair = tc.pair;
+
+  TcArgs t{};
+  TcMaps m{};
+  t.n_problems = n;
+  t.lr = a0.lr;
+  t.status = st;
+  t.lse_part = reinterpret_cast<float2*>(a0.lse_part);
+  t.lse = a0.lse; t.lse_sg = a0.lse_sg;
+  t.labels = a0.labels; t.labels_sg = a0.labels_sg;
+  t.label_logit = a0.label_logit;
+  t.inv_rows = a0.inv_rows;
+  int64_t tiles = 0;
+  int ks_first = 1;
+  for (int i = 0; i < n; ++i) {
+    const GemmArgs<bf16>& a = ga[i];
+    const int n_store = a.N_store > 0 ? a.N_store : a.N;
+    TcProblem& p = t.p[i];
+    p.M = a.M; p.N = n_store; p.K = a.K;
+    p.m_tiles = (int)ceil_div(a.M, BM * pair);
+    p.n_tiles = (int)ceil_div(n_store, bn);
+    p.G = a.G;
+    p.k_splits = 1;
+    p.kb_per_split = (int)ceil_div(a.K, BK);
+    if (a.k_splits > 1) {
+      if (a.epi != EPI_BIAS_F32 || a.bias) return false;   // slices are plain fp32 partial products
+      p.kb_per_split = (int)ceil_div(ceil_div(a.K, BK), a.k_splits);
+      p.k_splits = (int)ceil_div(ceil_div(a.K, BK), p.kb_per_split);
+      if (p.k_splits != a.k_splits) return false;           // caller sizes its buffer with gemm_tc_splits()
+    }
+    if (i == 0) ks_first = p.k_splits;
+    p.a_gmul = (a.G > 1 && a.a_sg != 0) ? 1 : 0;
+    p.b_gmul = (a.G > 1 && a.b_sg != 0) ? 1 : 0;
+    p.bias = a.bias; p.bias_sg = a.bias_sg;
+    tiles += (int64_t)p.m_tiles * p.n_tiles * p.G * p.k_splits;
+    if (tiles > 0x7fffffffll) return false;
+    p.tile_end = (int)tiles;
+    if (a.lr != a0.lr) return false;
+
+    // K-major operand: inner = K, outer = rows (M or N).  MN-major: inner = rows, outer = K.
+    const long long gga = p.a_gmul ? a.G : 1, ggb = p.b_gmul ? a.G : 1;
+    const bool ok_a = a_mn ? make_map(&m.a[i], a.A, 2, a.M, a.K, gga, a.a_sk, a.a_sg, 64, BK, 128)
+                           : make_map(&m.a[i], a.A, 2, a.K, a.M, gga, a.a_sm, a.a_sg, 64, BM, 128);
+    const bool ok_b = b_mn ? make_map(&m.b[i], a.B, 2, a.N, a.K, ggb, a.b_sk, a.b_sg, 64, BK, 128)
+                           : make_map(&m.b[i], a.B, 2, a.K, a.N, ggb, a.b_sn, a.b_sg, 64, bn / pair, 128);
+    if (!ok_a || !ok_b) return false;
+    m.c32[i] = m.a[i]; m.c16[i] = m.a[i]; m.aux16[i] = m.a[i];   // placeholders for the maps an epilogue does not use
+    // Output / epilogue-input chunks: [G][M][n_store] row-major, boxes of 128 rows x 32 columns.
+    switch (epi) {
+      case EPI_BIAS_RELU:
+        if (a_mn || !b_mn) return false;
+        if (!make_map(&m.c16[i], a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
+        break;
+      case EPI_BIAS_F32:
+        if (a_mn) return false;
+        if (!make_map(&m.c32[i], a.outf, 4, n_store, a.M, (long long)a.G * p.k_splits, a.outf_ld, a.outf_sg, CH, BM, 128))
+          return false;
+        break;
+      case EPI_LSE_PART:
+        if (a_mn || !b_mn || a.k_splits > 1 || !a.lse_part) return false;
+        break;
+      case EPI_SOFTMAX_DELTA:
+        if (a_mn || !b_mn || a.k_splits > 1 || !a.lse || !a.labels || !a.label_logit) return false;
+        if (!make_map(&m.c16[i], a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
+        break;
+      case EPI_RELU_MASK:
+        if (a_mn || b_mn) return false;
+        if (!make_map(&m.c16[i], a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
+        if (!make_map(&m.aux16[i], a.mask, 2, n_store, a.M, a.G, a.mask_ld, a.mask_sg, CH, BM, 64)) return false;
+        break;
+      case EPI_SGD:
+        if (!a_mn || !b_mn || !a.opw) return false;
+        if (!make_map(&m.c32[i], a.outf, 4, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 128)) return false;
+        if (!make_map(&m.c16[i], a.opw, 2, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 64)) return false;
+        break;
+      default:
+        return false;
+    }
+  }
+  t.total_tiles = (int)tiles;
+  if (chain) {
+    // Problem i + 1 reads problem i's output rows: same groups, same rows, hence the same tile rows.
+    // Every CTA of a unit stores ceil(N / 32) chunks per (group, tile row) and launch; the running
+    // totals are kept by the caller, who clears counters and totals together.
+    for (int i = 0; i + 1 < n; ++i) {
+      if (ga[i + 1].M != ga[i].M || ga[i + 1].G != ga[i].G || ga[i + 1].A != ga[i].out) return false;
+      unsigned* ctr = chain->counters + (size_t)i * chain->stride;
+      if ((size_t)t.p[i].G * t.p[i].m_tiles > chain->stride) return false;
+      chain->totals[i] += (unsigned)(pair * ceil_div(t.p[i].N, CH));
+      t.p[i].signal_ctr = ctr;
+      t.p[i + 1].wait_ctr = ctr;
+      t.p[i + 1].wait_target = chain->totals[i];
+    }
+  }
+  (void)ks_first;
+
+  switch (epi) {
     case EPI_BIAS_RELU:
-      if (a_mn || !b_mn) return false;
-      if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
       if (pair == 2) return launch<0, 1, 256, 6, 4, EPI_BIAS_RELU, 2>(L, m, t);
       if (bn == 256) return launch<0, 1, 256, 4, 4, EPI_BIAS_RELU, 1>(L, m, t);
       if (bn == 128) return launch<0, 1, 128, 6, 4, EPI_BIAS_RELU, 1>(L, m, t);
       return launch<0, 1, 64, 8, 4, EPI_BIAS_RELU, 1>(L, m, t);
     case EPI_BIAS_F32:
-      if (a_mn) return false;
-      if (!make_map(&m.c32, a.outf, 4, n_store, a.M, (long long)a.G * t.k_splits, a.outf_ld, a.outf_sg, CH, BM, 128))
-        return false;
       if (!a_mn && !b_mn) {   // both operands K-major: k slices of delta * W^T
         if (pair == 2) return launch<0, 0, 256, 6, 2, EPI_BIAS_F32, 2>(L, m, t);
         if (bn == 256) return launch<0, 0, 256, 4, 2, EPI_BIAS_F32, 1>(L, m, t);
@@ -992,32 +1172,23 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
       }
       // a short contraction (wide output layer fed by a narrow hidden layer) is bound by writing
       // the logits: fewer operand stages, a deeper ring of output chunks
-      if (pair == 2 && ceil_div(a.K, BK) <= 4) return launch<0, 1, 256, 3, 6, EPI_BIAS_F32, 2>(L, m, t);
+      if (pair == 2 && ceil_div(a0.K, BK) <= 4) return launch<0, 1, 256, 3, 6, EPI_BIAS_F32, 2>(L, m, t);
       if (pair == 2) return launch<0, 1, 256, 6, 2, EPI_BIAS_F32, 2>(L, m, t);
       if (bn == 256) return launch<0, 1, 256, 4, 2, EPI_BIAS_F32, 1>(L, m, t);
       if (bn == 128) return launch<0, 1, 128, 5, 4, EPI_BIAS_F32, 1>(L, m, t);
       return launch<0, 1, 64, 6, 4, EPI_BIAS_F32, 1>(L, m, t);
     case EPI_LSE_PART:
-      if (a_mn || !b_mn || a.k_splits > 1 || !a.lse_part) return false;
       if (pair == 2) return launch<0, 1, 256, 4, 1, EPI_LSE_PART, 2>(L, m, t);
       return launch<0, 1, 256, 3, 1, EPI_LSE_PART, 1>(L, m, t);
     case EPI_SOFTMAX_DELTA:
-      if (a_mn || !b_mn || a.k_splits > 1 || !a.lse || !a.labels || !a.label_logit) return false;
-      if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
       if (pair == 2) return launch<0, 1, 256, 4, 6, EPI_SOFTMAX_DELTA, 2>(L, m, t);
       return launch<0, 1, 256, 3, 6, EPI_SOFTMAX_DELTA, 1>(L, m, t);
     case EPI_RELU_MASK:
-      if (a_mn || b_mn) return false;
-      if (!make_map(&m.c16, a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
-      if (!make_map(&m.aux16, a.mask, 2, n_store, a.M, a.G, a.mask_ld, a.mask_sg, CH, BM, 64)) return false;
       if (pair == 2) return launch<0, 0, 256, 6, 4, EPI_RELU_MASK, 2>(L, m, t);
       if (bn == 256) return launch<0, 0, 256, 4, 4, EPI_RELU_MASK, 1>(L, m, t);
       if (bn == 128) return launch<0, 0, 128, 6, 4, EPI_RELU_MASK, 1>(L, m, t);
       return launch<0, 0, 64, 8, 4, EPI_RELU_MASK, 1>(L, m, t);
     case EPI_SGD:
-      if (!a_mn || !b_mn || !a.opw) return false;
-      if (!make_map(&m.c32, a.outf, 4, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 128)) return false;
-      if (!make_map(&m.c16, a.opw, 2, n_store, a.M, a.G, a.outf_ld, a.outf_sg, CH, BM, 64)) return false;
       if (pair == 2) return launch<1, 1, 256, 4, 4, EPI_SGD, 2>(L, m, t);
       if (bn == 128) return launch<1, 1, 128, 4, 4, EPI_SGD, 1>(L, m, t);
       return launch<1, 1, 64, 5, 4, EPI_SGD, 1>(L, m, t);
@@ -1025,5 +1196,7 @@ bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
       return false;
   }
 }
+
+bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) { return gemm_tc_batch(L, &a, 1, nullptr, st); }
 
 }  // namespace ist

@@ -27,7 +27,7 @@ struct Region {
 // Placement of everything that lives in the caller's workspace blob.
 struct Plan {
   size_t total = 0;
-  Region status, part, row_loss, logits, ev_a, ev_b, ev_acc, splitk, lse, label_logit;
+  Region status, part, row_loss, logits, ev_a, ev_b, ev_acc, splitk, lse, label_logit, chain_fwd, chain_dx;
   std::vector<Region> idx, off;             // hidden layer l at [l]  (1..t-1)
   std::vector<Region> master, bias, opw;    // layer l at [l]         (1..t)
   std::vector<Region> act, delta;           // act [0..t-1], delta [1..t]
@@ -74,6 +74,12 @@ struct ist_ctx {
 
   // subnets this context trains in ist_local_steps (all S unless ist_set_subnet_range narrowed it)
   int sub_first = 0, sub_count = 0;
+
+  // chained launches: running totals of the row-block counters (index = layer), and the batch size
+  // and subnet count they were accumulated with (a change clears counters and totals)
+  std::vector<unsigned> fwd_totals, dx_totals;
+  int chain_B = -1, chain_S = -1;
+  size_t chain_stride() const { return (size_t)S * ceil_div((int64_t)max_batch, 128); }
 
   // batch standardisation of hidden pre-activations (off unless ist_enable_normalization ran)
   bool norm = false, calibrated = false;
@@ -234,6 +240,10 @@ void make_plan(ist_ctx* c) {
       sk = std::max(sk, (size_t)(ks > 1 ? ks : 0) * S * Bm * c->ld[l - 1] * 4);
     }
   p.splitk = p.take(sk);
+  // row-block counters of chained launches (forward chain, delta chain): one set per layer
+  const size_t chain_words = (size_t)(t + 1) * S * ceil_div(Bm, 128);
+  p.chain_fwd = p.take(c->precision == IST_BF16 ? chain_words * 4 : 0);
+  p.chain_dx = p.take(c->precision == IST_BF16 ? chain_words * 4 : 0);
 }
 
 void make_norm_plan(ist_ctx* c) {
@@ -362,6 +372,31 @@ bool gemm(ist_ctx* c, const GemmArgs<float>& a) {
 }
 bool gemm(ist_ctx* c, const GemmArgs<bf16>& a) { return gemm_tc(c->launch(), a, c->status()); }
 
+// Several products of one kind in as few launches as possible.  fp32 operands: one CUDA-core
+// launch each.  bf16 operands: tiles of one tensor-core launch per gemm_tc_max_batch() problems;
+// with `chained`, every problem reads the output of the one before it and the launch orders
+// their tiles through the row-block counters of `region` (one set per problem, indexed by
+// `layer0 + i`; `totals` are the context's running sums for that region).
+bool gemm_list(ist_ctx* c, const std::vector<GemmArgs<float>>& v, bool, Region, std::vector<unsigned>*, int) {
+  for (auto& g : v) gemm_simt<float>(c->launch(), g);
+  return true;
+}
+bool gemm_list(ist_ctx* c, const std::vector<GemmArgs<bf16>>& v, bool chained, Region region,
+               std::vector<unsigned>* totals, int layer0) {
+  const int cap = gemm_tc_max_batch();
+  for (size_t i0 = 0; i0 < v.size(); i0 += cap) {
+    const int n = (int)std::min<size_t>(cap, v.size() - i0);
+    if (chained && n > 1) {
+      GemmChain ch{region.at<unsigned>(c->ws) + (size_t)(layer0 + i0) * c->chain_stride(), c->chain_stride(),
+                   totals->data() + layer0 + i0};
+      if (!gemm_tc_batch(c->launch(), v.data() + i0, n, &ch, c->status())) return false;
+    } else if (!gemm_tc_batch(c->launch(), v.data() + i0, n, nullptr, c->status())) {
+      return false;
+    }
+  }
+  return true;
+}
+
 // delta GEMM with the contraction cut into slices: fp32 partial slabs, then sum + ReLU mask.
 bool split_delta_gemm(ist_ctx*, const GemmArgs<float>&, int, int) { return false; }
 bool split_delta_gemm(ist_ctx* c, const GemmArgs<bf16>& masked, int want, int B) {
@@ -412,6 +447,16 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
   float* row_loss = c->plan.row_loss.at<float>(c->ws);
   DeviceStatus* st = c->status();
   Launch L = c->launch();
+  if (bf && (c->chain_B != B || c->chain_S != S)) {
+    // the counters' per-launch increments depend on the tile shape, which follows the batch
+    if (c->plan.chain_dx.offset > c->plan.chain_fwd.offset)
+      IST_CUDA(c, cudaMemsetAsync(c->plan.chain_fwd.at<char>(c->ws), 0,
+                                  2 * (c->plan.chain_dx.offset - c->plan.chain_fwd.offset), c->stream));
+    c->fwd_totals.assign(t + 2, 0u);
+    c->dx_totals.assign(t + 2, 0u);
+    c->chain_B = B;
+    c->chain_S = S;
+  }
 
   for (int k = 0; k < K; ++k) {
     const int64_t row0 = (int64_t)k * X->stride_step;
@@ -448,6 +493,17 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
                          c->nrstd(l), c->ld[l], act(l), Bm * c->ld[l]);
     };
     // ---- forward ---------------------------------------------------------------------------
+    // Hidden layers without standardisation form a chain a_l = relu(a_{l-1} W_l + b_l): they are
+    // collected and go out together (tiles of one launch, see gemm_list).
+    std::vector<GemmArgs<T>> fwd_chain;
+    int fwd_chain_l0 = 0;
+    auto flush_fwd = [&]() -> bool {
+      if (fwd_chain.empty()) return true;
+      Scope sc(c, IST_K_FWD);
+      const bool ok = gemm_list(c, fwd_chain, true, c->plan.chain_fwd, &c->fwd_totals, fwd_chain_l0);
+      fwd_chain.clear();
+      return ok;
+    };
     for (int l = 1; l <= t; ++l) {
       if (l == 1 && X->kind == IST_X_CSR && t > 1) {
         {
@@ -488,12 +544,19 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.epi = EPI_BIAS_F32;
         g.outf = logits; g.outf_ld = c->ld[t]; g.outf_sg = Bm * c->ld[t];
       }
+      if (g.epi == EPI_BIAS_RELU) {
+        if (fwd_chain.empty()) fwd_chain_l0 = l;
+        fwd_chain.push_back(g);
+        continue;
+      }
+      if (!flush_fwd()) return fail(c, IST_ERR_UNSUPPORTED, "forward GEMMs below layer %d cannot be launched", l);
       {
         Scope sc(c, IST_K_FWD);
         if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "forward GEMM of layer %d cannot be launched", l);
       }
       if (l < t && c->norm) standardise(l);
     }
+    if (!flush_fwd()) return fail(c, IST_ERR_UNSUPPORTED, "forward GEMMs cannot be launched");
     // ---- loss and its gradient -------------------------------------------------------------
     {
       Scope sc(c, IST_K_LOSS);
@@ -539,6 +602,15 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
     // Every delta is formed from the weights as they stood at the start of the step, so all of
     // them are computed first; the bias update follows at once, while the deltas it sums are still
     // in L2 (after the weight updates have streamed the masters through, they no longer are).
+    std::vector<GemmArgs<T>> dx_chain;      // delta_{l-1} = (delta_l W_l^T) * mask, l descending
+    int dx_chain_l0 = 0;
+    auto flush_dx = [&]() -> bool {
+      if (dx_chain.empty()) return true;
+      Scope sc(c, IST_K_DX);
+      const bool ok = gemm_list(c, dx_chain, true, c->plan.chain_dx, &c->dx_totals, dx_chain_l0);
+      dx_chain.clear();
+      return ok;
+    };
     for (int l = t; l > 1; --l) {
       {
         GemmArgs<T> g{};
@@ -549,13 +621,17 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.epi = EPI_RELU_MASK;
         g.mask = act(l - 1); g.mask_ld = c->ld[l - 1]; g.mask_sg = Bm * c->ld[l - 1];
         g.out = delta(l - 1); g.out_ld = c->ld[l - 1]; g.out_sg = Bm * c->ld[l - 1];
-        Scope sc(c, IST_K_DX);
         const int want = bf ? wanted_k_splits(c->np[l], c->np[l - 1], S, B) : 1;
         if (want > 1) {
+          if (!flush_dx()) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMMs above layer %d cannot be launched", l);
+          Scope sc(c, IST_K_DX);
           if (!split_delta_gemm(c, g, want, B))
             return fail(c, IST_ERR_UNSUPPORTED, "k-split delta GEMM of layer %d cannot be launched", l);
-        } else if (!gemm(c, g)) {
-          return fail(c, IST_ERR_UNSUPPORTED, "delta GEMM of layer %d cannot be launched", l);
+        } else {
+          if (dx_chain.empty()) dx_chain_l0 = t - l;
+          dx_chain.push_back(g);
+          if (c->norm && !flush_dx())
+            return fail(c, IST_ERR_UNSUPPORTED, "delta GEMM of layer %d cannot be launched", l);
         }
       }
       if (c->norm) {   // the masked product is d_zh; carry it through the standardisation
@@ -564,20 +640,17 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
                             c->nmu(l - 1), c->nrstd(l - 1), c->ld[l - 1], S, B, (int)c->np[l - 1]);
       }
     }
+    if (!flush_dx()) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMMs cannot be launched");
     // biases are not read by the backward pass, so their update may come before or after the
     // weight updates: before, if the deltas it sums are small enough to be still in L2 then
     size_t delta_bytes = 0;
     for (int l = 1; l <= t; ++l) delta_bytes += (size_t)S * B * c->ld[l] * sizeof(T);
     const bool bias_first = delta_bytes <= kL2ResidentBytes;
     if (bias_first) update_biases(t, 1);
+    // the weight updates of the dense layers do not depend on one another: tiles of one launch
+    std::vector<GemmArgs<T>> upd;
     for (int l = t; l >= 1; --l) {
-      if (l == 1 && X->kind == IST_X_CSR && t > 1) {
-        Scope sc(c, IST_K_SPMM);
-        spmm_backward_sgd<T>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
-                             delta(1), c->ld[1], Bm * c->ld[1], (int)c->np[1], master(1), opw(1),
-                             c->ld[1], c->slice_elems(1), lr);
-        continue;
-      }
+      if (l == 1 && X->kind == IST_X_CSR && t > 1) continue;
       GemmArgs<T> g{};
       g.M = (int)c->np[l - 1]; g.N = (int)c->np[l]; g.K = B; g.G = S;
       g.N_store = (int)c->ld[l];
@@ -587,8 +660,18 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       g.outf = master(l); g.outf_ld = c->ld[l]; g.outf_sg = c->slice_elems(l);
       g.opw = opw(l);
       g.lr = lr;
+      upd.push_back(g);
+    }
+    {
       Scope sc(c, IST_K_DW_SGD);
-      if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "weight-gradient GEMM of layer %d cannot be launched", l);
+      if (!gemm_list(c, upd, false, Region(), nullptr, 0))
+        return fail(c, IST_ERR_UNSUPPORTED, "weight-gradient GEMMs cannot be launched");
+    }
+    if (X->kind == IST_X_CSR && t > 1) {
+      Scope sc(c, IST_K_SPMM);
+      spmm_backward_sgd<T>(L, X->row_ptr, X->col, X->val, row0, X->stride_subnet, S, B, c->N[0],
+                           delta(1), c->ld[1], Bm * c->ld[1], (int)c->np[1], master(1), opw(1),
+                           c->ld[1], c->slice_elems(1), lr);
     }
     if (!bias_first) update_biases(t, 1);
   }

@@ -102,6 +102,20 @@ template <typename T> void gemm_simt(const Launch& L, const GemmArgs<T>& a);
 // Tensor-core path (tcgen05 + TMA) for bf16 operands.  Returns false if the shape cannot be
 // described to TMA (misaligned strides) or the operand layouts do not fit an epilogue.
 bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st);
+// Several products with the same operand layouts and epilogue (bias + ReLU, ReLU mask, or SGD
+// update) as tiles of one launch; at most gemm_tc_max_batch() of them, none k-split.  With a
+// chain, problem i + 1 must read problem i's output (A == out, same M and G) and its tiles wait for
+// the rows they read.  counters: device, [n - 1][stride] unsigned, stride >= G * ceil(M / 128);
+// totals: host, [n - 1], running sums this call advances.  The caller clears counters and totals
+// together (once at start, and whenever the batch's shape changes).  A chain must not be used
+// from two streams at once.
+struct GemmChain {
+  unsigned* counters;
+  size_t stride;
+  unsigned* totals;
+};
+bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* a, int n, const GemmChain* chain, DeviceStatus* st);
+int gemm_tc_max_batch();
 // Launches a one-block kernel whose bounded barrier wait must expire after limit_cycles (see
 // ist_selftest_wait_expiry).
 bool gemm_tc_wait_selftest(const Launch& L, DeviceStatus* st, long long limit_cycles);
