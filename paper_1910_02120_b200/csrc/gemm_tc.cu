@@ -213,6 +213,17 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* v) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 32 lanes x 16 consecutive 32-bit columns.
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 // Shared-memory matrix descriptor for a 128-byte-swizzled tile.
 //   bits  0..13 start address >> 4      bits 16..29 leading byte offset >> 4
 //   bits 32..45 stride byte offset >> 4 bits 46..47 descriptor version (1)
@@ -243,6 +254,9 @@ struct TcProblem {
   int k_splits, kb_per_split;   // the k range may be cut into slices that run as separate tiles
   int a_gmul, b_gmul;     // 1 if the operand has one slab per group, 0 if all groups share it
   int tile_end;
+  int head_f32;           // EPI_BIAS_RELU launches only: this problem writes plain fp32 products in
+                          // 16-column chunks through the c32 map (a narrow output layer riding on the
+                          // hidden layers' launch); 0 = the launch's ordinary epilogue
   const float* bias; long long bias_sg;
   // chaining: counters [G][m_tiles]; a tile of (g, mt) may load A once wait_ctr[g * m_tiles + mt]
   // has reached wait_target; a storer adds the chunks it has stored for (g, mt) to signal_ctr
@@ -370,7 +384,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
     for (int i = 0; i < a.n_problems; ++i) {
       prefetch_map(&maps.a[i]);
       prefetch_map(&maps.b[i]);
-      if (ET::k32) prefetch_map(&maps.c32[i]);
+      if (ET::k32 || (EPI == EPI_BIAS_RELU && a.p[i].head_f32)) prefetch_map(&maps.c32[i]);
       if (ET::k16) prefetch_map(&maps.c16[i]);
       if (EPI == EPI_RELU_MASK) prefetch_map(&maps.aux16[i]);
     }
@@ -581,6 +595,9 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
     for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
       const TileAt at = locate(a, tile, pi);
       const int pN = a.p[pi].N, pM = a.p[pi].M, p_ntiles = a.p[pi].n_tiles;
+      // a narrow fp32 head works in 16-column chunks: 128 x 16 floats fill the bf16 area of a slot
+      const bool head = EPI == EPI_BIAS_RELU && a.p[pi].head_f32;
+      const int cw = head ? CH / 2 : CH, nch = head ? 2 * NCH : NCH;
       const int n0 = at.nt * BN;
       const int g = at.slab;                          // output slab (group, k slice)
       const int b = j & 1;
@@ -601,8 +618,8 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
       if (!ok) break;
       tc_fence_after();
 #pragma unroll 1
-      for (int c = 0; c < NCH; ++c, ++cq) {
-        const int nc = n0 + c * CH;
+      for (int c = 0; c < nch; ++c, ++cq) {
+        const int nc = n0 + c * cw;
         if (nc >= pN) break;                          // CTA-uniform
         // A slot always belongs to the same warp group, so that the group sees the slot's barrier
         // phases in order (a parity wait cannot tell phase p from phase p + 2); every configuration
@@ -620,6 +637,17 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
           if (!ok) break;
         }
         uint32_t acc[32];
+        if (head) {
+          // plain product (a k slice of the logits; bias and the sum over slices come later)
+          tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * cw), acc);
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            *b16_unit(b16, r, u) = make_uint4(acc[4 * u], acc[4 * u + 1], acc[4 * u + 2], acc[4 * u + 3]);
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&chunk_done[slot]);
+          continue;
+        }
         tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * CH), acc);
         if (EPI == EPI_SGD) {
 #pragma unroll
@@ -784,8 +812,10 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         const int n0 = at.nt * BN;
         const int g = at.slab;
         unsigned stored = 0;                 // chunks of this tile this thread has stored
-        for (int c = 0; c < NCH; ++c, ++cq) {
-          const int nc = n0 + c * CH;
+        const bool head = EPI == EPI_BIAS_RELU && pr.head_f32;
+        const int cw = head ? CH / 2 : CH, nch = head ? 2 * NCH : NCH;
+        for (int c = 0; c < nch; ++c, ++cq) {
+          const int nc = n0 + c * cw;
           if (nc >= pr.N) break;
           const int slot = cq % NS;
           // a slot always belongs to the same storer, so that storer sees the slot's barrier
@@ -794,8 +824,12 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
           ok = mbar_wait(&chunk_done[slot], (cq / NS) & 1, abortp, a.status, 7);
           if (!ok) break;
           uint8_t* f32 = slots + slot * SLOT_BYTES;
-          if (ET::k32) tma_store_3d(&maps.c32[pi], f32, nc, m0, g);
-          if (ET::k16) tma_store_3d(&maps.c16[pi], f32 + F32_BYTES, nc, m0, g);
+          if (head) {
+            tma_store_3d(&maps.c32[pi], f32 + F32_BYTES, nc, m0, g);
+          } else {
+            if (ET::k32) tma_store_3d(&maps.c32[pi], f32, nc, m0, g);
+            if (ET::k16) tma_store_3d(&maps.c16[pi], f32 + F32_BYTES, nc, m0, g);
+          }
           tma_commit_group();
           ++stored;
           if (EPI == EPI_SGD && PAIR == 2) {
@@ -1048,13 +1082,21 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
   const GemmArgs<bf16>& a0 = ga[0];
   const int epi = a0.epi;
   const bool a_mn = a0.a_sm == 1 && a0.a_sk != 1, b_mn = a0.b_sn == 1 && a0.b_sk != 1;
+  // A narrow output layer may close a list of hidden forward layers: plain fp32 products (k slices
+  // allowed) of at most 64 columns, written in 16-column chunks by the same kernel instance.
+  const bool head = n > 1 && epi == EPI_BIAS_RELU && ga[n - 1].epi == EPI_BIAS_F32;
+  if (head) {
+    const GemmArgs<bf16>& h = ga[n - 1];
+    if (h.bias || !h.outf || (h.N_store > 0 ? h.N_store : h.N) > 64) return false;
+  }
   for (int i = 0; i < n; ++i) {
     const GemmArgs<bf16>& a = ga[i];
     const bool ai = a.a_sm == 1 && a.a_sk != 1, bi = a.b_sn == 1 && a.b_sk != 1;
-    if (a.epi != epi || ai != a_mn || bi != b_mn) return false;     // one kernel instance serves the batch
+    const bool is_head = head && i == n - 1;
+    if ((a.epi != epi && !is_head) || ai != a_mn || bi != b_mn) return false;   // one kernel instance serves the batch
     if (!ai && a.a_sk != 1) return false;
     if (!bi && a.b_sk != 1) return false;
-    if (n > 1 && a.k_splits > 1) return false;
+    if (n > 1 && a.k_splits > 1 && !is_head) return false;
   }
   if (n > 1 && epi != EPI_BIAS_RELU && epi != EPI_RELU_MASK && epi != EPI_SGD) return false;
   if (chain && (epi == EPI_SGD || n < 2 || !chain->counters || !chain->totals)) return false;
@@ -1074,7 +1116,6 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
   t.label_logit = a0.label_logit;
   t.inv_rows = a0.inv_rows;
   int64_t tiles = 0;
-  int ks_first = 1;
   for (int i = 0; i < n; ++i) {
     const GemmArgs<bf16>& a = ga[i];
     const int n_store = a.N_store > 0 ? a.N_store : a.N;
@@ -1085,13 +1126,14 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
     p.G = a.G;
     p.k_splits = 1;
     p.kb_per_split = (int)ceil_div(a.K, BK);
+    const bool is_head = head && i == n - 1;
+    p.head_f32 = is_head ? 1 : 0;
     if (a.k_splits > 1) {
       if (a.epi != EPI_BIAS_F32 || a.bias) return false;   // slices are plain fp32 partial products
       p.kb_per_split = (int)ceil_div(ceil_div(a.K, BK), a.k_splits);
       p.k_splits = (int)ceil_div(ceil_div(a.K, BK), p.kb_per_split);
       if (p.k_splits != a.k_splits) return false;           // caller sizes its buffer with gemm_tc_splits()
     }
-    if (i == 0) ks_first = p.k_splits;
     p.a_gmul = (a.G > 1 && a.a_sg != 0) ? 1 : 0;
     p.b_gmul = (a.G > 1 && a.b_sg != 0) ? 1 : 0;
     p.bias = a.bias; p.bias_sg = a.bias_sg;
@@ -1112,7 +1154,12 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
     switch (epi) {
       case EPI_BIAS_RELU:
         if (a_mn || !b_mn) return false;
-        if (!make_map(&m.c16[i], a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) return false;
+        if (is_head) {   // 128 x 16 fp32 chunks: 64-byte rows, like the bf16 chunks of the other problems
+          if (!make_map(&m.c32[i], a.outf, 4, n_store, a.M, (long long)a.G * p.k_splits, a.outf_ld, a.outf_sg, CH / 2, BM, 64))
+            return false;
+        } else if (!make_map(&m.c16[i], a.out, 2, n_store, a.M, a.G, a.out_ld, a.out_sg, CH, BM, 64)) {
+          return false;
+        }
         break;
       case EPI_BIAS_F32:
         if (a_mn) return false;
@@ -1155,7 +1202,6 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
       t.p[i + 1].wait_target = chain->totals[i];
     }
   }
-  (void)ks_first;
 
   switch (epi) {
     case EPI_BIAS_RELU:

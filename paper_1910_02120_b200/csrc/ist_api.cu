@@ -549,6 +549,12 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         fwd_chain.push_back(g);
         continue;
       }
+      // the k slices of a narrow output layer ride on the hidden layers' launch when there is room
+      if (bf && l == t && head && !fwd_chain.empty() && (int)fwd_chain.size() < gemm_tc_max_batch()) {
+        fwd_chain.push_back(g);
+        if (!flush_fwd()) return fail(c, IST_ERR_UNSUPPORTED, "forward GEMMs cannot be launched");
+        continue;
+      }
       if (!flush_fwd()) return fail(c, IST_ERR_UNSUPPORTED, "forward GEMMs below layer %d cannot be launched", l);
       {
         Scope sc(c, IST_K_FWD);
