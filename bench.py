@@ -29,10 +29,10 @@ from paper_1910_02120_b200 import synth  # noqa: E402
 
 METRIC = "IST training samples/sec (all S subnets, device-timed)"
 UNIT = "samples/s"
-# DRAM bytes per algorithmic byte, from ncu captures of the named class's main launch
-# (profiles/gemm_tc_C3.md).  Valid for the kernels as they stand in this file's revision; set an
-# entry to None when the kernel changes.
-NCU_TRAFFIC_RATIO = {"C3-wide-pixels": {"dw_sgd": 492.1 / 503.3, "fwd": None, "dx": None}}
+# DRAM bytes per launch from ncu captures, kept in a tracked file with the hash of the kernel
+# source each capture was taken on; a class whose source has changed since reports traffic = null.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
+CSRC = os.path.join(ROOT, "paper_1910_02120_b200", "csrc")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -77,6 +77,22 @@ def peaks():
     return p
 
 
+def measured_traffic(workload_name: str, kernel_class: str, work_per_launch_now: float):
+    """DRAM bytes per launch of this class from the recorded ncu capture, scaled by the launch's
+    algorithmic work in the record's unit (bytes for HBM-bound classes, flop for the contractions;
+    the capture may be of a reduced case of the same kernel), or None when there
+    is no capture for this workload and class or the kernel source has changed since."""
+    import hashlib
+    try:
+        rec = json.load(open(TRAFFIC_FILE))[workload_name][kernel_class]
+        src = open(os.path.join(CSRC, rec["source"]), "rb").read()
+    except (OSError, KeyError, ValueError):
+        return None
+    if hashlib.sha256(src).hexdigest() != rec["source_sha256"]:
+        return None
+    return rec["dram_bytes_per_launch"] * work_per_launch_now / rec["algorithmic_per_launch"]
+
+
 def config_dict(w: synth.Workload, n_gpus: int, norm_eps=None, sharded=False):
     extra = {} if norm_eps is None else {"normalization": f"per-neuron batch standardisation, eps={norm_eps:g}"}
     return {
@@ -97,7 +113,25 @@ def config_dict(w: synth.Workload, n_gpus: int, norm_eps=None, sharded=False):
 # algorithmic work per round (all S subnets), used for the roofline fractions
 # ---------------------------------------------------------------------------------------------
 
-def work_model(w: synth.Workload, norm=False):
+def spmm_bytes(w: synth.Workload, data, n1: int) -> float:
+    """Algorithmic bytes of the sparse first layer over a round (all subnets and local steps).
+    Forward, per stored nonzero and subnet: one bf16 weight row of n1 entries + 8 B (column and
+    value), and n1 * 2 B of output per batch row.  Backward with the fused update: per nonzero the
+    8 B again and the delta row (n1 * 2 B); per distinct touched input row 10 B per weight (fp32
+    master read and written, bf16 copy written)."""
+    es = 2 if w.precision == "bf16" else 4
+    total = 0.0
+    rp = np.asarray(data.row_ptr, dtype=np.int64)
+    for i in range(w.S * w.K):                       # one (subnet, step) minibatch each
+        lo, hi = rp[i * w.B], rp[(i + 1) * w.B]
+        nnz = float(hi - lo)
+        distinct = float(np.unique(data.col[lo:hi]).size)
+        total += nnz * (n1 * es + 8) + w.B * n1 * es            # forward
+        total += nnz * (8 + n1 * es) + distinct * n1 * (8 + (2 if es == 2 else 0))   # backward + update
+    return total
+
+
+def work_model(w: synth.Workload, norm=False, data=None):
     d, S, B, K = w.layer_dims, w.S, w.B, w.K
     t = len(d) - 1
     n = [d[0]] + [-(-d[l] // S) for l in range(1, t)] + [d[t]]
@@ -112,6 +146,8 @@ def work_model(w: synth.Workload, norm=False):
     hidden = B * S * sum(n[1:t])                    # hidden pre-activations per local step
     # standardisation: forward reads fp32 z and writes a; backward reads z and d_zh, writes d_z
     norm_bytes = {"norm": hidden * ((4 + es) + (4 + 2 * es)) * K} if norm else {}
+    if not dense_first and data is not None:
+        norm_bytes["spmm"] = spmm_bytes(w, data, n[1])
     return {
         "packed_elems": packed,
         "flops": {"fwd": fwd * K, "dx": dx * K, "dw_sgd": dw * K},
@@ -425,7 +461,7 @@ def run_ours(args, w):
         return
 
     pk = peaks()
-    wm = work_model(w, norm=args.norm_eps is not None)
+    wm = work_model(w, norm=args.norm_eps is not None, data=data if data.is_csr else None)
     if shard:      # this rank ran the local steps of its own subnets only; gather / scatter cover all S
         for k in ("fwd", "dx", "dw_sgd"):
             wm["flops"][k] = wm["flops"][k] * count // w.S
@@ -452,7 +488,8 @@ def run_ours(args, w):
     tensor_classes = ("fwd", "dx") if tensor_peak else ()
     if dominant in tensor_classes:
         roof = {"kernel": dominant, "bound": "tensor", "achieved": dk["tflops"], "peak": tensor_peak,
-                "unit": "TFLOP/s", "frac": dk["tflops"] / tensor_peak, "traffic": None,
+                "unit": "TFLOP/s", "frac": dk["tflops"] / tensor_peak,
+                "traffic": measured_traffic(w.name, dominant, wm["flops"][dominant] / dk["launches_per_step"]),
                 "peak_source": pk["_source"] + " (sustained bf16)",
                 "flops_per_launch": wm["flops"][dominant] / dk["launches_per_step"],
                 "avg_launch_ms": dk["ms_per_step"] / dk["launches_per_step"]}
@@ -461,8 +498,7 @@ def run_ours(args, w):
         roof = {"kernel": dominant, "bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": gbs / pk["hbm_gbs"], "peak_source": pk["_source"],
                 "bytes_per_launch": wm["bytes"][dominant] / dk["launches_per_step"],
-                "traffic": (NCU_TRAFFIC_RATIO.get(w.name, {}).get(dominant) or 0) * wm["bytes"][dominant] /
-                           dk["launches_per_step"] or None,
+                "traffic": measured_traffic(w.name, dominant, wm["bytes"][dominant] / dk["launches_per_step"]),
                 "avg_launch_ms": dk["ms_per_step"] / dk["launches_per_step"]}
     elif dominant in wm["flops"]:
         # fp32 CUDA-core contraction: 148 SMs x 128 FMA lanes x 2 flop x max clock

@@ -69,3 +69,24 @@ def test_reference_arm_is_silent_on_other_ranks():
     p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "C1",
                         "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=600, env=env)
     assert p.returncode == 0 and p.stdout.strip() == ""
+
+
+def test_recorded_dram_traffic_is_dropped_when_the_kernel_source_changes(tmp_path, monkeypatch):
+    """roofline.traffic comes from a tracked ncu record and must read null once the kernel it was
+    taken on has been edited."""
+    import hashlib
+    import json
+    import bench
+    src = tmp_path / "k.cu"
+    src.write_text("kernel v1")
+    rec = {"W": {"upd": {"dram_bytes_per_launch": 110.0, "algorithmic_per_launch": 100.0, "unit": "bytes",
+                         "source": "k.cu", "source_sha256": hashlib.sha256(b"kernel v1").hexdigest()}}}
+    f = tmp_path / "t.json"
+    f.write_text(json.dumps(rec))
+    monkeypatch.setattr(bench, "TRAFFIC_FILE", str(f))
+    monkeypatch.setattr(bench, "CSRC", str(tmp_path))
+    assert bench.measured_traffic("W", "upd", 200.0) == 220.0          # scaled by the launch's algorithmic work
+    assert bench.measured_traffic("W", "other", 200.0) is None
+    assert bench.measured_traffic("V", "upd", 200.0) is None
+    src.write_text("kernel v2")
+    assert bench.measured_traffic("W", "upd", 200.0) is None
