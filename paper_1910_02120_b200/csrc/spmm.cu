@@ -68,7 +68,13 @@ __global__ void spmm_forward_kernel(const int32_t* __restrict__ row_ptr, const i
   }
 }
 
-template <typename T>
+// Adds four floats to four adjacent words of global memory with one reduction instruction.
+__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
+  asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d)
+               : "memory");
+}
+
+template <typename T, bool VEC>
 __global__ void spmm_backward_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col,
                                      const float* __restrict__ val, int64_t row0,
                                      int64_t group_row_stride, int B, int64_t N0,
@@ -89,8 +95,14 @@ __global__ void spmm_backward_kernel(const int32_t* __restrict__ row_ptr, const 
     if (c < 0 || c >= N0) continue;   // reported by the forward pass
     float x = -lr * val[p];
     float* dst = Mg + (int64_t)c * p_ld;
+    if (VEC) {
+      // one 16-byte reduction per lane: the row segment is 16-byte aligned (p_ld % 4 == 0)
+      red_add_v4(dst, x * d[0], x * d[1], x * d[2], x * d[3]);
+    } else {
 #pragma unroll
-    for (int u = 0; u < 4; ++u) atomicAdd(dst + u, x * d[u]);
+      for (int u = 0; u < 4; ++u)
+        if (cc + u < d_ld) atomicAdd(dst + u, x * d[u]);
+    }
   }
 }
 
@@ -152,8 +164,12 @@ void spmm_backward_sgd(const Launch& L, const int32_t* row_ptr, const int32_t* c
                        const T* delta, int64_t d_ld, int64_t d_sg, int n1, float* master, bf16* opw,
                        int64_t p_ld, int64_t p_sg, float lr) {
   dim3 grid((unsigned)ceil_div(B, kRowsPerCta), G, (unsigned)ceil_div(d_ld, 128));
-  spmm_backward_kernel<T><<<grid, dim3(32, kRowsPerCta), 0, L.stream>>>(
-      row_ptr, col, val, row0, group_row_stride, B, N0, delta, d_ld, d_sg, master, p_ld, p_sg, lr);
+  if (p_ld % 4 == 0 && ((uintptr_t)master & 15) == 0 && p_sg % 4 == 0)
+    spmm_backward_kernel<T, true><<<grid, dim3(32, kRowsPerCta), 0, L.stream>>>(
+        row_ptr, col, val, row0, group_row_stride, B, N0, delta, d_ld, d_sg, master, p_ld, p_sg, lr);
+  else
+    spmm_backward_kernel<T, false><<<grid, dim3(32, kRowsPerCta), 0, L.stream>>>(
+        row_ptr, col, val, row0, group_row_stride, B, N0, delta, d_ld, d_sg, master, p_ld, p_sg, lr);
   L.count();
   if (opw) {
     spmm_refresh_kernel<<<grid, dim3(32, kRowsPerCta), 0, L.stream>>>(
