@@ -54,6 +54,8 @@ def parse_args():
                          "slices per round, strong scaling) instead of running N independent replicas")
     ap.add_argument("--norm-eps", type=float, default=None,
                     help="standardise hidden pre-activations over the batch (Sec. 2.2) with this epsilon")
+    ap.add_argument("--iid", action="store_true",
+                    help="independent assignment of neurons to subnets (unequal group sizes) instead of the balanced split")
     ap.add_argument("--local-steps", type=int, default=0,
                     help="override K (local steps per round); makes a small case for profiler captures")
     ap.add_argument("--sweep", action="store_true",
@@ -93,8 +95,10 @@ def measured_traffic(workload_name: str, kernel_class: str, work_per_launch_now:
     return rec["dram_bytes_per_launch"] * work_per_launch_now / rec["algorithmic_per_launch"]
 
 
-def config_dict(w: synth.Workload, n_gpus: int, norm_eps=None, sharded=False):
+def config_dict(w: synth.Workload, n_gpus: int, norm_eps=None, sharded=False, iid=False):
     extra = {} if norm_eps is None else {"normalization": f"per-neuron batch standardisation, eps={norm_eps:g}"}
+    if iid:
+        extra["partition"] = "independent assignment (unequal subnets)"
     return {
         **extra,
         "workload": f"{w.name}: MLP {'-'.join(map(str, w.layer_dims))}, S={w.S}, batch={w.B}, "
@@ -344,7 +348,8 @@ def run_ours(args, w):
             raise SystemExit("--shard-subnets takes dense inputs")
         data = synth.Batchset(y=data.y[first:first + count].copy(), X=data.X[first:first + count].copy())
     prec = api.IST_BF16 if w.precision == "bf16" else api.IST_FP32
-    ctx = api.Ist(w.layer_dims, w.S, prec, w.B, input_is_csr=data.is_csr, device=str(dev))
+    ctx = api.Ist(w.layer_dims, w.S, prec, w.B, input_is_csr=data.is_csr, device=str(dev),
+                  partition_rule=api.IST_PART_IID if args.iid else api.IST_PART_BALANCED)
     ctx.bind_weights(Wd, bd)
     if args.norm_eps is not None:
         ctx.enable_normalization(args.norm_eps)
@@ -406,7 +411,7 @@ def run_ours(args, w):
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                               "warmup": n_warm, "ms_per_step": ms / args.steps, "quick": True,
-                              "gpu_launches": launches, "config": config_dict(w, world, args.norm_eps, shard)}))
+                              "gpu_launches": launches, "config": config_dict(w, world, args.norm_eps, shard, args.iid)}))
         if world > 1:
             dist.destroy_process_group()
         return
@@ -516,7 +521,7 @@ def run_ours(args, w):
             ent["frac_of_hbm_peak"] = ent["gbs"] / pk["hbm_gbs"]
 
     cpu = None
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and not args.iid:
         smp = OracleSample(w, n_sub=2, norm_eps=args.norm_eps)
         t0 = time.perf_counter()
         vals = []
@@ -530,7 +535,7 @@ def run_ours(args, w):
         "warmup": n_warm, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "strong" if shard else "weak", "vs_baseline": None, "dtype": w.precision.replace("fp", "f"),
         "data": "synthetic",
-        "config": config_dict(w, world, args.norm_eps, shard), "clocks": clocks,
+        "config": config_dict(w, world, args.norm_eps, shard, args.iid), "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": launches, "roofline": roof, "kernels": kernels, "cpu_baseline": cpu,

@@ -254,6 +254,8 @@ struct TcProblem {
   int k_splits, kb_per_split;   // the k range may be cut into slices that run as separate tiles
   int a_gmul, b_gmul;     // 1 if the operand has one slab per group, 0 if all groups share it
   int tile_end;
+  // true extents of the groups (null: every group fills M / N / K), see GemmArgs
+  const int32_t* m_off; const int32_t* n_off; const int32_t* k_off;
   int head_f32;           // EPI_BIAS_RELU launches only: this problem writes plain fp32 products in
                           // 16-column chunks through the c32 map (a narrow output layer riding on the
                           // hidden layers' launch); 0 = the launch's ordinary epilogue
@@ -298,6 +300,20 @@ __device__ __forceinline__ TileAt locate(const TcArgs& a, int tile, int& pi) {
   t.nt = (lt / pr.m_tiles) % pr.n_tiles;
   t.slab = lt / (pr.m_tiles * pr.n_tiles);
   return t;
+}
+
+// Whether tile (mt, nt) of group g has any output inside the group's true extents, and how many
+// 64-deep k blocks its contraction really needs (at least one, so that the accumulator is
+// written: the operands beyond a group's depth are zeros).  Every role asks the same question
+// about every tile, so all of them skip the same tiles.
+template <int TILE_M, int TILE_N>
+__device__ __forceinline__ bool tile_live(const TcProblem& pr, const TileAt& at, int g, int* kb_limit) {
+  *kb_limit = 0x7fffffff;
+  if (!pr.m_off && !pr.n_off && !pr.k_off) return true;
+  if (pr.m_off && at.mt * TILE_M >= __ldg(pr.m_off + g + 1) - __ldg(pr.m_off + g)) return false;
+  if (pr.n_off && at.nt * TILE_N >= __ldg(pr.n_off + g + 1) - __ldg(pr.n_off + g)) return false;
+  if (pr.k_off) *kb_limit = max(1, (__ldg(pr.k_off + g + 1) - __ldg(pr.k_off + g) + BK - 1) / BK);
+  return true;
 }
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
@@ -447,7 +463,9 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         const int m0 = at.mt * (BM * PAIR) + rank * BM;     // this CTA's rows of A
         const int n0 = at.nt * BN + rank * BNL;             // this CTA's rows of B
         const int g = at.slab / pr.k_splits;
-        const int num_kb = (pr.K + BK - 1) / BK;
+        int kb_limit;
+        if (!tile_live<BM * PAIR, BN>(pr, at, g, &kb_limit)) continue;
+        const int num_kb = min((pr.K + BK - 1) / BK, kb_limit);
         const int kb0 = (at.slab % pr.k_splits) * pr.kb_per_split, kb1 = min(num_kb, kb0 + pr.kb_per_split);
         const int ga = g * pr.a_gmul, gb = g * pr.b_gmul;
         if (pr.wait_ctr) {
@@ -526,15 +544,17 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
       constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BN, BM * PAIR);
       int it = 0, j = 0, pi = 0;
       bool ok = true;
-      for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
+      for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
         const TileAt at = locate(a, tile, pi);
         const TcProblem& pr = a.p[pi];
+        int kb_limit;
+        if (!tile_live<BM * PAIR, BN>(pr, at, at.slab / pr.k_splits, &kb_limit)) continue;
         const int b = j & 1;
         ok = mbar_wait(&acc_empty[b], ((j >> 1) & 1) ^ 1, abortp, a.status, 2);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
-        const int num_kb = (pr.K + BK - 1) / BK;
+        const int num_kb = min((pr.K + BK - 1) / BK, kb_limit);
         const int kb0 = (at.slab % pr.k_splits) * pr.kb_per_split;
         const int kb1 = min(num_kb, kb0 + pr.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -558,6 +578,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         if (ok) {
           if (PAIR == 2) tc_commit_pair(&acc_full[b]); else tc_commit(&acc_full[b]);
         }
+        ++j;
       }
     }
   } else if (warp < kAuxWarp) {
@@ -592,8 +613,16 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
 #pragma unroll
     for (int c = 0; c < NCH; ++c) next_bias[c] = 0.f;
     if (unit < total_tiles) prefetch_tile_inputs(unit);
-    for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++j) {
+    for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
       const TileAt at = locate(a, tile, pi);
+      {
+        int kb_limit;
+        if (!tile_live<BM * PAIR, BN>(a.p[pi], at, at.slab / a.p[pi].k_splits, &kb_limit)) {
+          // the inputs requested for this tile are dropped; ask for the next tile's
+          if (tile + n_units < total_tiles) prefetch_tile_inputs(tile + n_units);
+          continue;
+        }
+      }
       const int pN = a.p[pi].N, pM = a.p[pi].M, p_ntiles = a.p[pi].n_tiles;
       // a narrow fp32 head works in 16-column chunks: 128 x 16 floats fill the bf16 area of a slot
       const bool head = EPI == EPI_BIAS_RELU && a.p[pi].head_f32;
@@ -769,6 +798,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
       if (lane == 0) {   // the accumulator is free again: tell the CTA that issues the MMAs
         if (PAIR == 2) mbar_arrive_cluster(map_to_cta(&acc_empty[b], 0)); else mbar_arrive(&acc_empty[b]);
       }
+      ++j;
     }
   } else if (warp == kAuxWarp) {
     // ---------------------------------------------------------------- epilogue input loads
@@ -777,6 +807,10 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
         const TileAt at = locate(a, tile, pi);
+        {
+          int kb_limit;
+          if (!tile_live<BM * PAIR, BN>(a.p[pi], at, at.slab / a.p[pi].k_splits, &kb_limit)) continue;
+        }
         const int pN = a.p[pi].N;
         const int m0 = at.mt * (BM * PAIR) + rank * BM;
         const int n0 = at.nt * BN;
@@ -808,6 +842,19 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
         const TileAt at = locate(a, tile, pi);
         const TcProblem& pr = a.p[pi];
+        {
+          int kb_limit;
+          if (!tile_live<BM * PAIR, BN>(pr, at, at.slab / pr.k_splits, &kb_limit)) {
+            // A skipped tile still counts towards its row block, so that the rows' readers wait for
+            // the same total whatever the group's extent (they never read behind the extent).
+            if (pr.signal_ctr && sj == 0) {
+              const int live = min(NCH, (pr.N - at.nt * BN + CH - 1) / CH);
+              if (live > 0)
+                red_release_add(pr.signal_ctr + (long long)(at.slab / pr.k_splits) * pr.m_tiles + at.mt, (unsigned)live);
+            }
+            continue;
+          }
+        }
         const int m0 = at.mt * (BM * PAIR) + rank * BM;
         const int n0 = at.nt * BN;
         const int g = at.slab;
@@ -1137,6 +1184,8 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
     p.a_gmul = (a.G > 1 && a.a_sg != 0) ? 1 : 0;
     p.b_gmul = (a.G > 1 && a.b_sg != 0) ? 1 : 0;
     p.bias = a.bias; p.bias_sg = a.bias_sg;
+    p.m_off = a.m_off; p.n_off = a.n_off; p.k_off = a.k_off;
+    if (a.k_off && p.k_splits > 1) return false;
     tiles += (int64_t)p.m_tiles * p.n_tiles * p.G * p.k_splits;
     if (tiles > 0x7fffffffll) return false;
     p.tile_end = (int)tiles;

@@ -406,6 +406,7 @@ bool split_delta_gemm(ist_ctx* c, const GemmArgs<bf16>& masked, int want, int B)
   g.epi = EPI_BIAS_F32;
   g.bias = nullptr;
   g.k_splits = ks;
+  g.n_off = nullptr; g.k_off = nullptr;   // every slice writes its whole slab: the reduction reads all of it
   g.outf = part; g.outf_ld = masked.out_ld; g.outf_sg = (int64_t)B * masked.out_ld;
   g.out = nullptr; g.mask = nullptr;
   if (!gemm_tc(c->launch(), g, c->status())) return false;
@@ -445,6 +446,11 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
   };
   float* logits = c->plan.logits.at<float>(c->ws);
   float* row_loss = c->plan.row_loss.at<float>(c->ws);
+  // Unequal subnets (independent assignment): the group offsets of hidden layer l tell the
+  // tensor-core launches each group's true extent; null for the input / output layers and under the
+  // balanced rule, where every group fills its slab (up to one neuron).
+  const bool ragged = c->rule == IST_PART_IID && bf;
+  auto off_of = [&](int l) -> const int32_t* { return (ragged && l >= 1 && l < t) ? c->off(l) + s0 : nullptr; };
   DeviceStatus* st = c->status();
   Launch L = c->launch();
   if (bf && (c->chain_B != B || c->chain_S != S)) {
@@ -526,6 +532,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       g.A = in_ptr(l - 1); g.a_sm = in_ld(l - 1); g.a_sk = 1; g.a_sg = in_sg(l - 1);
       g.B = weights(l); g.b_sn = 1; g.b_sk = c->ld[l]; g.b_sg = c->slice_elems(l);
       g.bias = bias_of(l); g.bias_sg = c->ld[l];
+      g.n_off = off_of(l); g.k_off = off_of(l - 1);
       if (l < t && c->norm) {
         g.epi = EPI_BIAS_F32;        // fp32 pre-activations; standardisation and ReLU follow
         g.outf = c->zbuf(l); g.outf_ld = c->ld[l]; g.outf_sg = Bm * c->ld[l];
@@ -539,6 +546,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.epi = EPI_BIAS_F32;        // k slices of the logits; bias and the sum happen in the softmax kernel
         g.bias = nullptr;
         g.k_splits = head_ks;
+        if (head_ks > 1) g.k_off = nullptr;
         g.outf = logits; g.outf_ld = c->ld[t]; g.outf_sg = (int64_t)B * c->ld[t];
       } else {
         g.epi = EPI_BIAS_F32;
@@ -574,6 +582,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.A = in_ptr(t - 1); g.a_sm = in_ld(t - 1); g.a_sk = 1; g.a_sg = in_sg(t - 1);
         g.B = weights(t); g.b_sn = 1; g.b_sk = c->ld[t]; g.b_sg = c->slice_elems(t);
         g.bias = bias_of(t); g.bias_sg = c->ld[t];
+        g.k_off = off_of(t - 1);
         g.epi = EPI_SOFTMAX_DELTA;
         g.out = delta(t); g.out_ld = c->ld[t]; g.out_sg = Bm * c->ld[t];
         g.lse = lse; g.lse_sg = Bm;
@@ -624,6 +633,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
         g.N_store = (int)c->ld[l - 1];
         g.A = delta(l); g.a_sm = c->ld[l]; g.a_sk = 1; g.a_sg = Bm * c->ld[l];
         g.B = weights(l); g.b_sn = c->ld[l]; g.b_sk = 1; g.b_sg = c->slice_elems(l);
+        g.n_off = off_of(l - 1); g.k_off = off_of(l);
         g.epi = EPI_RELU_MASK;
         g.mask = act(l - 1); g.mask_ld = c->ld[l - 1]; g.mask_sg = Bm * c->ld[l - 1];
         g.out = delta(l - 1); g.out_ld = c->ld[l - 1]; g.out_sg = Bm * c->ld[l - 1];
@@ -662,6 +672,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       g.N_store = (int)c->ld[l];
       g.A = in_ptr(l - 1); g.a_sm = 1; g.a_sk = in_ld(l - 1); g.a_sg = in_sg(l - 1);
       g.B = delta(l); g.b_sn = 1; g.b_sk = c->ld[l]; g.b_sg = Bm * c->ld[l];
+      g.m_off = off_of(l - 1); g.n_off = off_of(l);
       g.epi = EPI_SGD;
       g.outf = master(l); g.outf_ld = c->ld[l]; g.outf_sg = c->slice_elems(l);
       g.opw = opw(l);

@@ -83,6 +83,12 @@ struct GemmArgs {
                 // partial product to outf slab g * k_splits + s (EPI_BIAS_F32 without bias only)
   const T* A; int64_t a_sm, a_sk, a_sg;
   const T* B; int64_t b_sn, b_sk, b_sg;
+  // Per-group extents (tensor-core path; device pointers or null): group g really has
+  // off[g + 1] - off[g] rows (m_off), columns (n_off) or contraction entries (k_off); M, N, K are
+  // then the capacity every group is laid out for, and the rest of a slab holds zeros.  Tiles
+  // that lie wholly beyond a group's rows or columns are skipped and contractions stop at the
+  // group's depth (unequal subnets: work follows the true shapes, not the padded ones).
+  const int32_t* m_off; const int32_t* n_off; const int32_t* k_off;
   int epi;
   const float* bias; int64_t bias_sg;
   T* out; int64_t out_ld, out_sg;

@@ -87,3 +87,28 @@ def test_iid_slices_and_untouched_round_are_exact():
     ctx.sync_status()
     for l in range(len(W)):
         assert np.array_equal(Wd[l].cpu().numpy(), W[l]) and np.array_equal(bd[l].cpu().numpy(), b[l])
+
+
+@pytest.mark.parametrize("precision,dims,S,B", [("bf16", [64, 700, 520, 12], 3, 96), ("bf16", [256, 4096, 4096, 16], 8, 512)])
+def test_iid_two_rounds_with_changing_group_sizes(precision, dims, S, B):
+    """Unequal subnets work on their true shapes: tiles beyond a group's extent are skipped, so the
+    buffers behind them keep values from the round before, when the group may have been larger.
+    Two rounds with different draws must still follow the oracle."""
+    w = _wl(dims, S, B, 2, precision, lr=0.01)
+    W, b, data = H.make_problem(w, bias_scale=0.1)
+    from oracle import ist_oracle as O
+    o = O.IstOracle(w.layer_dims, w.S, partition_rule="iid")
+    o.bind_weights(W, b)
+    ctx, Wd, bd = H.gpu_context(w, W, b, rule="iid")
+    X, y = H.gpu_inputs(w, data)
+    sizes = []
+    for seed in (11, 12):
+        oloss = o.round(seed, data.X, data.y, w.lr, w.K)
+        gloss = ctx.round(seed, X, y, w.lr, w.K, w.B).cpu().numpy()
+        ctx.sync_status()
+        sizes.append([np.diff(p[1]).tolist() for p in o.parts])
+        assert abs(gloss.mean() - oloss.mean()) <= 1e-3
+        for l in range(len(W)):
+            H.assert_close(Wd[l].cpu().numpy(), o.W[l], 2e-2, f"W_{l + 1} after seed {seed}")
+            H.assert_close(bd[l].cpu().numpy(), o.b[l], 2e-2, f"b_{l + 1} after seed {seed}")
+    assert sizes[0] != sizes[1]
