@@ -69,6 +69,72 @@ __global__ void scatter_kernel(float* __restrict__ W, SliceMap m, const float* _
   }
 }
 
+// ---- last layer: whole rows, picked by the previous hidden layer's partition --------------------
+// W_t[G_{t-1}^s, :] keeps every column, so both sides are contiguous along a row and the kernel is a
+// strided row copy.  Rows of the full matrix start at any 4-byte offset (N_t is arbitrary), hence
+// scalar accesses; a thread keeps kRowU x kColU of them in flight (consecutive lanes on
+// consecutive columns), which is what the copy needs to approach the DRAM rate.
+constexpr int kRowU = 4, kColU = 4;
+
+template <bool GATHER>
+__global__ void __launch_bounds__(kThreads) rows_kernel(float* __restrict__ W, SliceMap m, float* __restrict__ master,
+                                                         bf16* __restrict__ opw) {
+  const int s = m.s_first + blockIdx.z;
+  const int nrows = m.row_off[s + 1] - m.row_off[s];
+  const int32_t* rows = m.row_idx + m.row_off[s];
+  const int64_t j0 = (int64_t)blockIdx.x * (kThreads * kColU) + threadIdx.x;
+  for (int64_t i0 = (int64_t)blockIdx.y * kRowU; i0 < (GATHER ? m.rows_pad : nrows); i0 += (int64_t)gridDim.y * kRowU) {
+    float v[kRowU][kColU];
+    int64_t src[kRowU];
+#pragma unroll
+    for (int u = 0; u < kRowU; ++u) src[u] = (i0 + u < nrows) ? (int64_t)rows[i0 + u] * m.full_cols : -1;
+    if (GATHER) {
+#pragma unroll
+      for (int u = 0; u < kRowU; ++u)
+#pragma unroll
+        for (int c = 0; c < kColU; ++c) {
+          const int64_t j = j0 + c * kThreads;
+          v[u][c] = (src[u] >= 0 && j < m.full_cols) ? __ldg(W + src[u] + j) : 0.f;   // pad rows / columns are zeros
+        }
+#pragma unroll
+      for (int u = 0; u < kRowU; ++u)
+#pragma unroll
+        for (int c = 0; c < kColU; ++c) {
+          const int64_t j = j0 + c * kThreads;
+          if (i0 + u < m.rows_pad && j < m.ld) {
+            const int64_t o = ((int64_t)s * m.rows_pad + i0 + u) * m.ld + j;
+            master[o] = v[u][c];
+            if (opw) opw[o] = __float2bfloat16_rn(v[u][c]);
+          }
+        }
+    } else {
+#pragma unroll
+      for (int u = 0; u < kRowU; ++u)
+#pragma unroll
+        for (int c = 0; c < kColU; ++c) {
+          const int64_t j = j0 + c * kThreads;
+          v[u][c] = (src[u] >= 0 && j < m.full_cols) ? __ldg(master + ((int64_t)s * m.rows_pad + i0 + u) * m.ld + j) : 0.f;
+        }
+#pragma unroll
+      for (int u = 0; u < kRowU; ++u)
+#pragma unroll
+        for (int c = 0; c < kColU; ++c) {
+          const int64_t j = j0 + c * kThreads;
+          if (src[u] >= 0 && j < m.full_cols) W[src[u] + j] = v[u][c];
+        }
+    }
+  }
+}
+
+bool rows_ok(const SliceMap& m) { return m.row_idx && !m.col_idx && m.full_cols >= 1024; }
+
+template <bool GATHER>
+void launch_rows(const Launch& L, float* W, const SliceMap& m, int S, float* master, bf16* opw) {
+  dim3 grid((unsigned)ceil_div(m.ld, kThreads * kColU), (unsigned)std::min<int64_t>(ceil_div(m.rows_pad, kRowU), 65535), S);
+  rows_kernel<GATHER><<<grid, kThreads, 0, L.stream>>>(W, m, master, opw);
+  L.count();
+}
+
 // ---- first layer: a column permutation, staged through shared memory -------------------------
 // W_1[:, G_1^s] keeps whole rows and permutes their columns.  A CTA stages kStageRows rows x
 // kStageCols consecutive columns (coalesced float4 accesses on the full-matrix side); because
@@ -307,6 +373,7 @@ __global__ void copy_out_kernel(const float* __restrict__ packed, int64_t ld, in
 void gather_slices(const Launch& L, const float* W, const SliceMap& m, int S, float* master,
                    bf16* opw, DeviceStatus* st) {
   if (staged_ok(m, S) && launch_permute_cols<true>(L, const_cast<float*>(W), m, S, master, opw, st)) return;
+  if (rows_ok(m)) return launch_rows<true>(L, const_cast<float*>(W), m, S, master, opw);
   dim3 grid((unsigned)ceil_div(m.ld, kThreads), (unsigned)std::min<int64_t>(ceil_div(m.rows_pad, kRowsPerCta), 65535), S);
   gather_kernel<<<grid, kThreads, 0, L.stream>>>(W, m, master, opw);
   L.count();
@@ -315,6 +382,7 @@ void gather_slices(const Launch& L, const float* W, const SliceMap& m, int S, fl
 void scatter_slices(const Launch& L, float* W, const SliceMap& m, int S, const float* master,
                     DeviceStatus* st) {
   if (staged_ok(m, S) && launch_permute_cols<false>(L, W, m, S, const_cast<float*>(master), nullptr, st)) return;
+  if (rows_ok(m)) return launch_rows<false>(L, W, m, S, const_cast<float*>(master), nullptr);
   dim3 grid((unsigned)ceil_div(m.ld, kThreads), (unsigned)std::min<int64_t>(ceil_div(m.rows_pad, kRowsPerCta), 65535), S);
   scatter_kernel<<<grid, kThreads, 0, L.stream>>>(W, m, master);
   L.count();
