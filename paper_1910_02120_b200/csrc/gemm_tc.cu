@@ -18,6 +18,9 @@
 //   warps 11..14 (one lane each) TMA stores of finished slots (coalesced, clipped at the tensor
 //                      edge); slot i belongs to storer i % 4, which hands the slot back as soon
 //                      as its own store has read it, without waiting for a later chunk
+//   warps 15..16       weight-update launches on single CTAs only: column sums of the B operand (the
+//                      deltas) as its k-slabs pass through shared memory, which is the bias
+//                      gradient; the bias update then needs no pass of its own over the deltas
 // The epilogue has no CTA-wide barrier: slots move between loader, epilogue warps and storer
 // through mbarriers (slot_full -> chunk_done -> slot_empty), so warps work on different chunks
 // at the same time and a slow chunk does not hold the others back.
@@ -63,7 +66,10 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;                   // 64 bf16 = 128 bytes = one swizzle row
 constexpr int CH = 32;                   // epilogue chunk: 32 output columns
-constexpr int kThreads = 480;            // 15 warps, see the role list above
+constexpr int kThreads = 480;            // 15 warps, see the role list above; the weight-update launches add two
+constexpr int kSumWarps = 2;
+constexpr bool sums_in_kernel(int epi, int pair) { return epi == 3 /* EPI_SGD */ && pair == 1; }
+constexpr int threads_for(int epi, int pair) { return kThreads + (sums_in_kernel(epi, pair) ? kSumWarps * 32 : 0); }
 constexpr int kEpiWarps = 8;
 constexpr int kAuxWarp = 10;
 constexpr int kStoreWarp0 = 11, kStoreWarps = 4;
@@ -256,6 +262,8 @@ struct TcProblem {
   int tile_end;
   // true extents of the groups (null: every group fills M / N / K), see GemmArgs
   const int32_t* m_off; const int32_t* n_off; const int32_t* k_off;
+  // weight-update launches: bias[g * bias_upd_sg + n] -= lr * sum_k B[g](n, k) for n < bias_n (null: none)
+  float* bias_upd; long long bias_upd_sg; int bias_n;
   int head_f32;           // EPI_BIAS_RELU launches only: this problem writes plain fp32 products in
                           // 16-column chunks through the c32 map (a narrow output layer riding on the
                           // hidden layers' launch); 0 = the launch's ordinary epilogue
@@ -269,6 +277,10 @@ struct TcProblem {
 struct TcArgs {
   int n_problems, total_tiles;
   TcProblem p[kMaxProblems];
+  // weight-update launches: the step's mean losses, loss.loss_out[g * out_stride + k] = mean of
+  // loss.row_loss[g][0 .. loss_B) for g < loss_G (loss_out null: none)
+  LossReduce loss;
+  int loss_B, loss_G;
   float lr;
   DeviceStatus* status;
   // wide softmax head (see GemmArgs); single-problem launches only
@@ -306,12 +318,20 @@ __device__ __forceinline__ TileAt locate(const TcArgs& a, int tile, int& pi) {
 // 64-deep k blocks its contraction really needs (at least one, so that the accumulator is
 // written: the operands beyond a group's depth are zeros).  Every role asks the same question
 // about every tile, so all of them skip the same tiles.
+// Weight-update launches on single CTAs: the tiles of the first tile row also sum their column
+// block's deltas for the bias update.
+__device__ __forceinline__ bool sums_bias(const TcProblem& pr, const TileAt& at) {
+  return pr.bias_upd != nullptr && at.mt == 0;
+}
+
 template <int TILE_M, int TILE_N>
 __device__ __forceinline__ bool tile_live(const TcProblem& pr, const TileAt& at, int g, int* kb_limit) {
   *kb_limit = 0x7fffffff;
   if (!pr.m_off && !pr.n_off && !pr.k_off) return true;
-  if (pr.m_off && at.mt * TILE_M >= __ldg(pr.m_off + g + 1) - __ldg(pr.m_off + g)) return false;
   if (pr.n_off && at.nt * TILE_N >= __ldg(pr.n_off + g + 1) - __ldg(pr.n_off + g)) return false;
+  // a tile that carries its columns' bias update runs even if it lies beyond the group's rows
+  if (pr.m_off && at.mt * TILE_M >= __ldg(pr.m_off + g + 1) - __ldg(pr.m_off + g) && !sums_bias(pr, at))
+    return false;
   if (pr.k_off) *kb_limit = max(1, (__ldg(pr.k_off + g + 1) - __ldg(pr.k_off + g) + BK - 1) / BK);
   return true;
 }
@@ -369,7 +389,7 @@ __device__ __forceinline__ uint4* b16_unit(uint8_t* area, int r, int u) {
 }
 
 template <int A_MN, int B_MN, int BN, int STAGES, int NS, int EPI, int PAIR>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(threads_for(EPI, PAIR), 1)
 gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcArgs a) {
   using ET = EpiTraits<EPI>;
   constexpr int BNL = BN / PAIR;   // rows of the B tile this CTA loads
@@ -381,6 +401,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
   constexpr uint32_t TMEM_COLS = 2 * BN;
   constexpr int NCH = BN / CH;
   constexpr bool kStore = ET::k32 || ET::k16;   // the epilogue writes chunks through the slot ring
+  constexpr bool kSums = sums_in_kernel(EPI, PAIR);   // two more warps sum the deltas for the bias update
   constexpr float kLog2e = 1.4426950408889634f;
 
   extern __shared__ uint8_t smem_raw[];
@@ -388,6 +409,8 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
   uint8_t* slots = smem + STAGES * STAGE_BYTES;
   __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
   __shared__ uint64_t slot_full[NS], chunk_done[NS], slot_empty[NS];
+  // weight update on single CTAs: "stage is full" passed on to the summing warps, and their "stage has been read"
+  __shared__ uint64_t stage_here[STAGES], sum_done[STAGES];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
@@ -408,7 +431,9 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], 1);
+      mbar_init(&stage_here[s], 1);
+      mbar_init(&empty_bar[s], 1);                 // the MMA commit
+      mbar_init(&sum_done[s], kSumWarps);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&acc_full[b], 1);
@@ -454,6 +479,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
     // ---------------------------------------------------------------- operand loads
     if (lane == 0) {
       int it = 0, pi = 0;
+      uint32_t sum_pending = 0, sum_parity = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
         const TileAt at = locate(a, tile, pi);
@@ -486,10 +512,22 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
           if (!ok) break;
           fence_proxy_async_all();
         }
+        const bool sums = kSums && sums_bias(pr, at);   // the summing warps read this tile's B stages
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           ok = mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abortp, a.status, 1);
           if (!ok) break;
+          if (kSums) {
+            // a stage that a summing tile filled last is free once the summing warps have read it
+            // too; they signal per stage, so bit s of sum_parity is the phase to wait for next
+            if ((sum_pending >> s) & 1u) {
+              ok = mbar_wait(&sum_done[s], (sum_parity >> s) & 1u, abortp, a.status, 12);
+              if (!ok) break;
+              sum_parity ^= 1u << s;
+              sum_pending &= ~(1u << s);
+            }
+            if (sums) sum_pending |= 1u << s;
+          }
           uint8_t* sa = smem + s * STAGE_BYTES;
           uint8_t* sb = sa + A_BYTES;
           if (PAIR == 2) {
@@ -542,7 +580,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
     // ---------------------------------------------------------------- MMA issue
     if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BN, BM * PAIR);
-      int it = 0, j = 0, pi = 0;
+      int it = 0, j = 0, pi = 0, sit = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
         const TileAt at = locate(a, tile, pi);
@@ -557,11 +595,19 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         const int num_kb = min((pr.K + BK - 1) / BK, kb_limit);
         const int kb0 = (at.slab % pr.k_splits) * pr.kb_per_split;
         const int kb1 = min(num_kb, kb0 + pr.kb_per_split);
+        const bool sums = kSums && sums_bias(pr, at);   // the summing warps follow this tile
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           ok = mbar_wait(&full_bar[s], (it / STAGES) & 1, abortp, a.status, 3);
           if (!ok) break;
           tc_fence_after();
+          if (kSums && sums) {
+            // tell the summing warps that the stage is full; they have a ring of their own,
+            // stepped once per stage of a summing tile, so that its phases stay in step with
+            // them although they skip the other tiles
+            mbar_arrive(&stage_here[sit % STAGES]);
+            ++sit;
+          }
           const uint32_t sa = smem_u32(smem + s * STAGE_BYTES), sb = sa + A_BYTES;
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
@@ -574,6 +620,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
           }
           // frees the slot (in both CTAs of a pair) once these MMAs have read it
           if (PAIR == 2) tc_commit_pair(&empty_bar[s]); else tc_commit(&empty_bar[s]);
+
         }
         if (ok) {
           if (PAIR == 2) tc_commit_pair(&acc_full[b]); else tc_commit(&acc_full[b]);
@@ -909,6 +956,85 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
       tma_wait_all();                // all stores complete before the CTA exits
     }
   }
+  if (kSums && warp >= kStoreWarp0 + kStoreWarps) {
+    // ---------------------------------------------------------------- bias gradient (and loss means)
+    // Summing warp sw owns the 64-column box sw of the B tile (MN-major: row k of a box holds 64
+    // consecutive columns, 128 bytes, 16-byte units swizzled by k % 8); lane l adds up columns
+    // 8 (l % 8) .. + 7 over the rows k = l / 8 (mod 4), and the four lanes of a column combine
+    // their sums at the end of the tile.  Only the first tile row carries a bias update
+    // (sums_bias); the summing warps step over the stages of all other tiles.  A stage of a
+    // summing tile is released by the MMA commit and by both summing warps (sum_done, which the
+    // loading thread waits for before it refills such a stage).  The MMA thread, which sees every
+    // stage fill up, passes the completions of a summing tile on through the stage_here ring.
+    // The ring is stepped once per stage of a summing tile and the MMA thread cannot be STAGES
+    // steps ahead (refilling a stage needs the summing warps' arrival), so a parity wait on it
+    // is unambiguous, which one on full_bar would not be for warps that skip tiles.
+    const int sw = warp - (kStoreWarp0 + kStoreWarps);
+    if (rank == 0 && sw == kSumWarps - 1 && a.loss.loss_out) {
+      for (int g = unit; g < a.loss_G; g += n_units) {
+        float acc = 0.f;
+        for (int b = lane; b < a.loss_B; b += 32) acc += __ldg(a.loss.row_loss + (long long)g * a.loss_B + b);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) a.loss.loss_out[(long long)g * a.loss.out_stride + a.loss.k] = acc / (float)a.loss_B;
+      }
+    }
+    constexpr int kBoxes = BNL / 64;
+    static_assert(!kSums || kBoxes <= kSumWarps, "one summing warp per 64-column box");
+    int it = 0, pi = 0, sit = 0;
+    bool ok = true;
+    for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
+      const TileAt at = locate(a, tile, pi);
+      const TcProblem& pr = a.p[pi];
+      int kb_limit;
+      if (!tile_live<BM * PAIR, BN>(pr, at, at.slab, &kb_limit)) continue;
+      const int num_kb = min((pr.K + BK - 1) / BK, kb_limit);
+      if (!sums_bias(pr, at)) {
+        it += num_kb;
+        continue;
+      }
+      const bool sum = sw < kBoxes;
+      const int u = lane & 7, rq = lane >> 3;   // this lane's 16-byte unit (8 columns) and row quarter
+      float acc[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+      for (int kb = 0; kb < num_kb; ++kb, ++it, ++sit) {
+        const int s = it % STAGES;
+        const uint32_t par = (sit / STAGES) & 1;
+        ok = mbar_wait(&stage_here[sit % STAGES], par, abortp, a.status, 10);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (sum) {
+          // one instruction reads four rows of the box (512 contiguous bytes, every bank once)
+          const uint8_t* box = smem + s * STAGE_BYTES + A_BYTES + sw * (BK * 128);
+#pragma unroll
+          for (int i = 0; i < BK / 4; ++i) {
+            const int k = 4 * i + rq;
+            float v[8];
+            unpack8(*reinterpret_cast<const uint4*>(box + k * 128 + ((u ^ (k & 7)) << 4)), v);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] += v[e];
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sum_done[s]);
+      }
+      if (ok && sum) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {             // the four row quarters of a column, in a fixed order
+          acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 8);
+          acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);
+        }
+        if (rq == 0) {
+          const int n = at.nt * BN + rank * BNL + sw * 64 + 8 * u;
+          float* bp = pr.bias_upd + (long long)at.slab * pr.bias_upd_sg + n;
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            if (n + e < pr.bias_n) bp[e] -= a.lr * acc[e];
+        }
+      }
+    }
+  }
   tc_fence_before();
   __syncthreads();
   if (PAIR == 2) cluster_sync_all();   // neither CTA leaves while the other may still touch its memory
@@ -1031,7 +1157,7 @@ bool launch(const Launch& L, const TcMaps& m, const TcArgs& t) {
     if (PAIR == 2) {
       cudaLaunchConfig_t probe{};
       probe.gridDim = dim3(2 * (sm_count() / 2));
-      probe.blockDim = dim3(kThreads);
+      probe.blockDim = dim3(threads_for(EPI, PAIR));
       probe.dynamicSmemBytes = smem;
       cudaLaunchAttribute attr{};
       attr.id = cudaLaunchAttributeClusterDimension;
@@ -1050,7 +1176,7 @@ bool launch(const Launch& L, const TcMaps& m, const TcArgs& t) {
   const int units = total < max_units ? total : max_units;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(PAIR * units);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(threads_for(EPI, PAIR));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = L.stream;
   cudaLaunchAttribute attrs[2];
@@ -1121,10 +1247,17 @@ int gemm_tc_splits(int K, int want) {
 
 int gemm_tc_max_batch() { return kMaxProblems; }
 
+// Whether a weight-update launch of these products would run on single CTAs, whose extra warps
+// can sum the deltas for the bias update (GemmArgs::bias_upd) and reduce the step's losses.
+bool gemm_tc_update_sums_bias(const GemmArgs<bf16>* a, int n) {
+  return n >= 1 && n <= kMaxProblems && pick_tile(a, n, EPI_SGD).pair == 1;
+}
+
 // Counters a chain of n problems over G groups and up to max_rows output rows needs.
 size_t gemm_tc_chain_counters(int n, int G, int max_rows) { return (size_t)n * G * ceil_div(max_rows, BM); }
 
-bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmChain* chain, DeviceStatus* st) {
+bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmChain* chain, const LossReduce* loss,
+                   DeviceStatus* st) {
   if (n < 1 || n > kMaxProblems) return false;
   const GemmArgs<bf16>& a0 = ga[0];
   const int epi = a0.epi;
@@ -1162,6 +1295,12 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
   t.labels = a0.labels; t.labels_sg = a0.labels_sg;
   t.label_logit = a0.label_logit;
   t.inv_rows = a0.inv_rows;
+  if (loss && (epi != EPI_SGD || pair != 1)) return false;
+  if (loss) {
+    t.loss = *loss;
+    t.loss_B = a0.K;          // the contraction of a weight update runs over the batch
+    t.loss_G = a0.G;
+  }
   int64_t tiles = 0;
   for (int i = 0; i < n; ++i) {
     const GemmArgs<bf16>& a = ga[i];
@@ -1185,6 +1324,8 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
     p.b_gmul = (a.G > 1 && a.b_sg != 0) ? 1 : 0;
     p.bias = a.bias; p.bias_sg = a.bias_sg;
     p.m_off = a.m_off; p.n_off = a.n_off; p.k_off = a.k_off;
+    if (a.bias_upd && (epi != EPI_SGD || pair != 1)) return false;   // see gemm_tc_update_sums_bias
+    p.bias_upd = a.bias_upd; p.bias_upd_sg = a.bias_upd_sg; p.bias_n = a.bias_n;
     if (a.k_off && p.k_splits > 1) return false;
     tiles += (int64_t)p.m_tiles * p.n_tiles * p.G * p.k_splits;
     if (tiles > 0x7fffffffll) return false;
@@ -1292,6 +1433,8 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
   }
 }
 
-bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) { return gemm_tc_batch(L, &a, 1, nullptr, st); }
+bool gemm_tc(const Launch& L, const GemmArgs<bf16>& a, DeviceStatus* st) {
+  return gemm_tc_batch(L, &a, 1, nullptr, nullptr, st);
+}
 
 }  // namespace ist

@@ -377,20 +377,30 @@ bool gemm(ist_ctx* c, const GemmArgs<bf16>& a) { return gemm_tc(c->launch(), a, 
 // with `chained`, every problem reads the output of the one before it and the launch orders
 // their tiles through the row-block counters of `region` (one set per problem, indexed by
 // `layer0 + i`; `totals` are the context's running sums for that region).
-bool gemm_list(ist_ctx* c, const std::vector<GemmArgs<float>>& v, bool, Region, std::vector<unsigned>*, int) {
+bool gemm_list(ist_ctx* c, const std::vector<GemmArgs<float>>& v, bool, Region, std::vector<unsigned>*, int,
+               const LossReduce* = nullptr) {
   for (auto& g : v) gemm_simt<float>(c->launch(), g);
   return true;
 }
+// Whether every launch a weight-update list is cut into can sum the deltas for the bias update.
+bool update_sums_bias(const std::vector<GemmArgs<float>>&) { return false; }
+bool update_sums_bias(const std::vector<GemmArgs<bf16>>& v) {
+  const int cap = gemm_tc_max_batch();
+  for (size_t i0 = 0; i0 < v.size(); i0 += cap)
+    if (!gemm_tc_update_sums_bias(v.data() + i0, (int)std::min<size_t>(cap, v.size() - i0))) return false;
+  return !v.empty();
+}
+// `loss` (weight-update lists only): the first launch also reduces the step's mean losses.
 bool gemm_list(ist_ctx* c, const std::vector<GemmArgs<bf16>>& v, bool chained, Region region,
-               std::vector<unsigned>* totals, int layer0) {
+               std::vector<unsigned>* totals, int layer0, const LossReduce* loss = nullptr) {
   const int cap = gemm_tc_max_batch();
   for (size_t i0 = 0; i0 < v.size(); i0 += cap) {
     const int n = (int)std::min<size_t>(cap, v.size() - i0);
     if (chained && n > 1) {
       GemmChain ch{region.at<unsigned>(c->ws) + (size_t)(layer0 + i0) * c->chain_stride(), c->chain_stride(),
                    totals->data() + layer0 + i0};
-      if (!gemm_tc_batch(c->launch(), v.data() + i0, n, &ch, c->status())) return false;
-    } else if (!gemm_tc_batch(c->launch(), v.data() + i0, n, nullptr, c->status())) {
+      if (!gemm_tc_batch(c->launch(), v.data() + i0, n, &ch, nullptr, c->status())) return false;
+    } else if (!gemm_tc_batch(c->launch(), v.data() + i0, n, nullptr, i0 == 0 ? loss : nullptr, c->status())) {
       return false;
     }
   }
@@ -600,10 +610,10 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
     }
     // ---- backward + SGD, last layer first --------------------------------------------------
     // db_l = sum_b delta_l, layers l_lo..l_hi; the step's mean losses are reduced by the same launch
-    auto update_biases = [&](int l_hi, int l_lo) {
+    auto update_biases = [&](int l_hi, int l_lo, bool with_loss = true) {
       Scope sc(c, IST_K_BIAS_SGD);
       BiasSgdArgs<T> ba{};
-      LossReduce lo{row_loss, loss_out, K, k};
+      LossReduce lo{row_loss, with_loss ? loss_out : nullptr, K, k};
       int n = 0;
       for (int l = l_hi; l >= l_lo; --l) {
         ba.layer[n++] = BiasSgdLayer<T>{delta(l), c->ld[l], Bm * c->ld[l], bias_of(l), c->ld[l], (int)c->np[l]};
@@ -657,12 +667,6 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       }
     }
     if (!flush_dx()) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMMs cannot be launched");
-    // biases are not read by the backward pass, so their update may come before or after the
-    // weight updates: before, if the deltas it sums are small enough to be still in L2 then
-    size_t delta_bytes = 0;
-    for (int l = 1; l <= t; ++l) delta_bytes += (size_t)S * B * c->ld[l] * sizeof(T);
-    const bool bias_first = delta_bytes <= kL2ResidentBytes;
-    if (bias_first) update_biases(t, 1);
     // the weight updates of the dense layers do not depend on one another: tiles of one launch
     std::vector<GemmArgs<T>> upd;
     for (int l = t; l >= 1; --l) {
@@ -679,9 +683,31 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       g.lr = lr;
       upd.push_back(g);
     }
+    // Biases are not read by the backward pass, so their update may come before or after the
+    // weight updates.  While the deltas it sums are small enough to be still in L2, the bias
+    // kernel runs first and costs next to nothing.  Deltas beyond that size (a very wide output
+    // layer) would be read from memory a second time: there the weight-update launch, when it
+    // runs on single CTAs, sums the deltas it streams anyway (its B operand), updates the biases
+    // itself and reduces the step's mean losses; what is left for the bias kernel is a sparse
+    // first layer's bias.  Otherwise the bias kernel runs last.
+    const bool sparse_first = X->kind == IST_X_CSR && t > 1;
+    size_t delta_bytes = 0;
+    for (int l = 1; l <= t; ++l) delta_bytes += (size_t)S * B * c->ld[l] * sizeof(T);
+    const bool bias_first = delta_bytes <= kL2ResidentBytes;
+    const bool bias_in_gemm = !bias_first && update_sums_bias(upd);
+    if (bias_in_gemm) {
+      for (auto& g : upd) {
+        const int l = (int)(&g - upd.data());   // upd[i] is layer t - i
+        g.bias_upd = bias_of(t - l); g.bias_upd_sg = c->ld[t - l]; g.bias_n = (int)c->np[t - l];
+      }
+      if (sparse_first) update_biases(1, 1, false);
+    } else if (bias_first) {
+      update_biases(t, 1);
+    }
     {
       Scope sc(c, IST_K_DW_SGD);
-      if (!gemm_list(c, upd, false, Region(), nullptr, 0))
+      LossReduce lo{row_loss, loss_out, K, k};
+      if (!gemm_list(c, upd, false, Region(), nullptr, 0, (bias_in_gemm && loss_out) ? &lo : nullptr))
         return fail(c, IST_ERR_UNSUPPORTED, "weight-gradient GEMMs cannot be launched");
     }
     if (X->kind == IST_X_CSR && t > 1) {
@@ -690,7 +716,7 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
                            delta(1), c->ld[1], Bm * c->ld[1], (int)c->np[1], master(1), opw(1),
                            c->ld[1], c->slice_elems(1), lr);
     }
-    if (!bias_first) update_biases(t, 1);
+    if (!bias_in_gemm && !bias_first) update_biases(t, 1);
   }
   IST_CUDA(c, cudaGetLastError());
   return IST_OK;

@@ -89,6 +89,10 @@ struct GemmArgs {
   // that lie wholly beyond a group's rows or columns are skipped and contractions stop at the
   // group's depth (unequal subnets: work follows the true shapes, not the padded ones).
   const int32_t* m_off; const int32_t* n_off; const int32_t* k_off;
+  // EPI_SGD on the tensor-core path, launches on single CTAs only (gemm_tc_update_sums_bias): the
+  // launch also updates the layer's bias from the B operand (the deltas) it streams anyway:
+  // bias_upd[g * bias_upd_sg + n] -= lr * sum_k B[g](n, k), n < bias_n.
+  float* bias_upd; int64_t bias_upd_sg; int bias_n;
   int epi;
   const float* bias; int64_t bias_sg;
   T* out; int64_t out_ld, out_sg;
@@ -120,8 +124,13 @@ struct GemmChain {
   size_t stride;
   unsigned* totals;
 };
-bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* a, int n, const GemmChain* chain, DeviceStatus* st);
+// loss (weight-update launches on single CTAs only, may be null): the step's mean losses are
+// reduced by the launch.
+struct LossReduce;
+bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* a, int n, const GemmChain* chain, const LossReduce* loss,
+                   DeviceStatus* st);
 int gemm_tc_max_batch();
+bool gemm_tc_update_sums_bias(const GemmArgs<bf16>* a, int n);
 // Launches a one-block kernel whose bounded barrier wait must expire after limit_cycles (see
 // ist_selftest_wait_expiry).
 bool gemm_tc_wait_selftest(const Launch& L, DeviceStatus* st, long long limit_cycles);
