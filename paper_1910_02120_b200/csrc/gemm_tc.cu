@@ -10,16 +10,20 @@
 //   warp 0 (one lane)  TMA loads of the A / B k-slabs into a ring of STAGES slots
 //   warp 1 (one lane)  tcgen05.mma issue; owns the tensor-memory allocation (2 accumulators,
 //                      so the MMAs of tile i+1 overlap the epilogue of tile i)
-//   warps 2..9         epilogue, two groups of four warps that take alternate 32-column chunks:
+//   then the epilogue warps, groups of four that take the 32-column chunks in turn (two groups;
+//                      four for the softmax passes over a very wide output layer):
 //                      tcgen05.ld (warp w reads lanes 32*(w%4)..+31, one row per thread), apply
 //                      the epilogue, write the chunk into a swizzled shared-memory slot
-//   warp 10 (one lane) TMA loads of the epilogue's input chunks into the slots: the fp32 master
-//                      slice for the SGD update, the ReLU mask for the delta GEMM
-//   warps 11..14 (one lane each) TMA stores of finished slots (coalesced, clipped at the tensor
-//                      edge); slot i belongs to storer i % 4, which hands the slot back as soon
-//                      as its own store has read it, without waiting for a later chunk
-//   warps 15..16       weight-update launches on single CTAs only: column sums of the B operand (the
-//                      deltas) as its k-slabs pass through shared memory, which is the bias
+//   then one warp (one lane), where the epilogue has input chunks: their TMA loads into the
+//                      slots (the fp32 master slice for the SGD update, the ReLU mask for the
+//                      delta GEMM)
+//   then the storers (one lane each; four, two beside sixteen epilogue warps, none where the
+//                      epilogue stores no chunks): TMA stores of finished slots (coalesced,
+//                      clipped at the tensor edge); slot i belongs to storer i % (their number),
+//                      which hands the slot back as soon as its own store has read it, without
+//                      waiting for a later chunk
+//   then two warps, weight-update launches on single CTAs only: column sums of the B operand
+//                      (the deltas) as its k-slabs pass through shared memory, which is the bias
 //                      gradient; the bias update then needs no pass of its own over the deltas
 // The epilogue has no CTA-wide barrier: slots move between loader, epilogue warps and storer
 // through mbarriers (slot_full -> chunk_done -> slot_empty), so warps work on different chunks
@@ -66,13 +70,20 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;                   // 64 bf16 = 128 bytes = one swizzle row
 constexpr int CH = 32;                   // epilogue chunk: 32 output columns
-constexpr int kThreads = 480;            // 15 warps, see the role list above; the weight-update launches add two
+// Warps of a CTA, see the role list above: loader, MMA issuer, the epilogue warps (two groups of
+// four; four groups for the two softmax passes over a very wide output layer, whose epilogues are
+// long chains of dependent instructions and need more warps to hide them), the epilogue input
+// loader, four storers, and two summing warps for weight-update launches on single CTAs.
 constexpr int kSumWarps = 2;
 constexpr bool sums_in_kernel(int epi, int pair) { return epi == 3 /* EPI_SGD */ && pair == 1; }
-constexpr int threads_for(int epi, int pair) { return kThreads + (sums_in_kernel(epi, pair) ? kSumWarps * 32 : 0); }
-constexpr int kEpiWarps = 8;
-constexpr int kAuxWarp = 10;
-constexpr int kStoreWarp0 = 11, kStoreWarps = 4;
+constexpr int epi_warps(int epi) { return (epi == 5 /* EPI_LSE_PART */ || epi == 6 /* EPI_SOFTMAX_DELTA */) ? 16 : 8; }
+constexpr bool has_aux(int epi) { return epi == 2 /* EPI_RELU_MASK */ || epi == 3; }   // EpiTraits::kAux
+// storers: none where the epilogue stores no chunks (EpiTraits::k32 || k16), two beside sixteen
+// epilogue warps (20 warps leave a thread 96 registers, 22 would leave 80), else four
+constexpr int store_warps(int epi) { return epi == 5 ? 0 : epi == 6 ? 2 : 4; }
+constexpr int threads_for(int epi, int pair) {
+  return (2 + epi_warps(epi) + (has_aux(epi) ? 1 : 0) + store_warps(epi) + (sums_in_kernel(epi, pair) ? kSumWarps : 0)) * 32;
+}
 constexpr long long kWaitLimitCycles = 2000000000ll;   // ~1 s at 2 GHz
 constexpr uint32_t kSuspendHintNs = 20000;             // a waiting thread may sleep this long inside one try_wait
 
@@ -144,8 +155,20 @@ __device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
   return r;
 }
+// Arrival on a barrier of another CTA of the cluster, which hands back a tensor-memory
+// accumulator whose reads have completed (tcgen05.wait::ld, then
+// tcgen05.fence::before_thread_sync); no data in memory goes with it.  CLUSTER_SCOPE: release at
+// cluster scope, which stalls the arriving warp for most of a microsecond per tile; otherwise
+// the instruction's default, release at CTA scope.  The softmax passes over a very wide output
+// layer, whose tiles are short, take the cheap form (C4: the two passes 2.4 -> 2.2 ms per local
+// step); the weight update measured 4 % slower with it than with the stall and keeps the
+// cluster scope, as do the other epilogues, where it makes no difference.
+template <bool CLUSTER_SCOPE>
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+  if (CLUSTER_SCOPE)
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+  else
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -256,6 +279,7 @@ constexpr int kMaxProblems = 4;
 // One product of a launch.  Tiles tile_end(previous) .. tile_end - 1 of the flat list are its.
 struct TcProblem {
   int M, N, K;            // M, N: bounds of the output rows / columns the epilogue touches
+  int n_true;             // columns of the product proper (<= N; the rest pads the rows): the softmax passes count only these
   int m_tiles, n_tiles, G;
   int k_splits, kb_per_split;   // the k range may be cut into slices that run as separate tiles
   int a_gmul, b_gmul;     // 1 if the operand has one slab per group, 0 if all groups share it
@@ -402,6 +426,12 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
   constexpr int NCH = BN / CH;
   constexpr bool kStore = ET::k32 || ET::k16;   // the epilogue writes chunks through the slot ring
   constexpr bool kSums = sums_in_kernel(EPI, PAIR);   // two more warps sum the deltas for the bias update
+  static_assert(EPI_RELU_MASK == 2 && EPI_SGD == 3 && EPI_LSE_PART == 5 && EPI_SOFTMAX_DELTA == 6 &&
+                    has_aux(EPI) == ET::kAux && (store_warps(EPI) > 0) == kStore,
+                "the role layout functions name epilogues by value");
+  constexpr int kEpiWarps = epi_warps(EPI), NG = kEpiWarps / 4;   // epilogue warps; groups of four
+  // first warp after the epilogue warps: the input loader if the epilogue has one, then the storers
+  constexpr int kAuxWarp = 2 + kEpiWarps, kStoreWarp0 = kAuxWarp + (ET::kAux ? 1 : 0), kStoreWarps = store_warps(EPI);
   constexpr float kLog2e = 1.4426950408889634f;
 
   extern __shared__ uint8_t smem_raw[];
@@ -441,7 +471,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
     }
     for (int s = 0; s < NS; ++s) {
       mbar_init(&slot_full[s], 1);               // loader's TMA bytes
-      mbar_init(&chunk_done[s], kEpiWarps / 2);  // the four warps that worked on the chunk
+      mbar_init(&chunk_done[s], 4);              // the four warps that worked on the chunk
       mbar_init(&slot_empty[s], 1);              // storer: the store has read the slot
     }
     abort_flag = 0;
@@ -631,10 +661,11 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
   } else if (warp < kAuxWarp) {
     // ---------------------------------------------------------------- epilogue
     const int q = warp & 3;                           // tensor-memory lane quarter of this warp
-    const int wg = (warp - 2) >> 2;                   // this warp's group takes chunks with cq % 2 == wg
+    const int wg = (warp - 2) >> 2;                   // this warp's group takes chunks with cq % NG == wg
     const int r = q * 32 + lane;                      // row of the tile owned by this thread
     int cq = 0, j = 0, pi = 0, pi_next = 0;
     bool ok = true;
+    float run_max = -INFINITY;                        // EPI_LSE_PART: the reference exponent, see there
     // per-tile epilogue inputs, requested one tile ahead (see below)
     float next_bias[NCH];
     float next_lse = 0.f;
@@ -643,13 +674,19 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
       const TileAt at = locate(a, tile, pi_next);
       const TcProblem& pr = a.p[pi_next];
       const int n0 = at.nt * BN;
-      if (EPI == EPI_BIAS_RELU || EPI == EPI_BIAS_F32 || EPI == EPI_LSE_PART || EPI == EPI_SOFTMAX_DELTA) {
+      if (EPI == EPI_BIAS_RELU || EPI == EPI_BIAS_F32) {
         const float* bias = pr.bias ? pr.bias + (long long)(at.slab / pr.k_splits) * pr.bias_sg : nullptr;
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           const int n = n0 + c * CH + lane;
           next_bias[c] = (bias && n < pr.N) ? __ldg(bias + n) : 0.f;
         }
+      }
+      if (EPI == EPI_LSE_PART || EPI == EPI_SOFTMAX_DELTA) {
+        // the softmax passes read the chunk's bias values straight from memory (warp-uniform
+        // 16-byte loads): one warp asks for the next tile's eight lines into L1 a tile ahead
+        if (warp == 2 && lane < BN * 4 / 128 && pr.bias && n0 + 32 * lane < pr.N)
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(pr.bias + (long long)at.slab * pr.bias_sg + n0 + 32 * lane));
       }
       if (EPI == EPI_SOFTMAX_DELTA) {
         const int row = at.mt * (BM * PAIR) + rank * BM + r;
@@ -670,7 +707,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
           continue;
         }
       }
-      const int pN = a.p[pi].N, pM = a.p[pi].M, p_ntiles = a.p[pi].n_tiles;
+      const int pN = a.p[pi].N, pNt = a.p[pi].n_true, pM = a.p[pi].M, p_ntiles = a.p[pi].n_tiles;
       // a narrow fp32 head works in 16-column chunks: 128 x 16 floats fill the bf16 area of a slot
       const bool head = EPI == EPI_BIAS_RELU && a.p[pi].head_f32;
       const int cw = head ? CH / 2 : CH, nch = head ? 2 * NCH : NCH;
@@ -685,8 +722,9 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
 #pragma unroll
       for (int c = 0; c < NCH; ++c) bias_reg[c] = next_bias[c];
       const int row = at.mt * (BM * PAIR) + rank * BM + r;   // this thread's row of the output
-      float run_max = -INFINITY, run_sum = 0.f;       // EPI_LSE_PART: over this warp group's chunks
-      const float row_lse = next_lse * kLog2e;        // log-sum-exp in the log2 domain
+      float run_sum = 0.f;                            // EPI_LSE_PART: over this warp group's chunks of the tile
+      // softmax pass: log-sum-exp in the log2 domain, with the division by the batch size folded in
+      const float row_lse = EPI == EPI_SOFTMAX_DELTA ? next_lse * kLog2e - log2f(a.inv_rows) : 0.f;
       const int row_label = next_label;
       if (tile + n_units < total_tiles) prefetch_tile_inputs(tile + n_units);
       // warp-uniform outcome: the tensor-memory loads below need the whole warp
@@ -699,9 +737,9 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         if (nc >= pN) break;                          // CTA-uniform
         // A slot always belongs to the same warp group, so that the group sees the slot's barrier
         // phases in order (a parity wait cannot tell phase p from phase p + 2); every configuration
-        // that stores through the ring has an even number of slots, so the groups alternate.
-        static_assert(!kStore || NS % 2 == 0, "slot ring needs an even number of slots");
-        if ((cq & 1) != wg) continue;
+        // that stores through the ring has a multiple of NG slots, so the groups take turns.
+        static_assert(!kStore || NS % NG == 0, "slot ring: a whole number of slots per warp group");
+        if ((cq % NG) != wg) continue;
         const int slot = cq % NS;
         uint8_t* f32 = slots + slot * SLOT_BYTES;
         uint8_t* b16 = f32 + F32_BYTES;
@@ -755,46 +793,73 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
             *pm = pack8(o);
           }
         } else if (EPI == EPI_LSE_PART || EPI == EPI_SOFTMAX_DELTA) {
-          // Both passes work on z * log2(e), so that every exponential is one ex2 and the scaling
-          // rides on the multiply-add that also adds the bias.
-          float bl = 0.f;
-#pragma unroll
-          for (int i = 0; i < NCH; ++i)
-            if (i == c) bl = bias_reg[i];
-          bl *= kLog2e;
+          // z = C + bias; every exponential is one ex2 of z * log2(e) minus a per-row constant,
+          // which is the multiply-add that follows the bias addition.  The bias values of the
+          // chunk are the same for every row: warp-uniform 16-byte loads, served by L1.
           float z[32];
+          {
+            const float* bias = a.p[pi].bias ? a.p[pi].bias + (long long)g * a.p[pi].bias_sg + nc : nullptr;
 #pragma unroll
-          for (int e = 0; e < 32; ++e)
-            z[e] = fmaf(__uint_as_float(acc[e]), kLog2e, __shfl_sync(0xffffffffu, bl, e));
+            for (int u = 0; u < 8; ++u) {
+              const float4 bv = (bias && nc + 4 * u < pN) ? __ldg(reinterpret_cast<const float4*>(bias) + u)
+                                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+              z[4 * u + 0] = __uint_as_float(acc[4 * u + 0]) + bv.x;
+              z[4 * u + 1] = __uint_as_float(acc[4 * u + 1]) + bv.y;
+              z[4 * u + 2] = __uint_as_float(acc[4 * u + 2]) + bv.z;
+              z[4 * u + 3] = __uint_as_float(acc[4 * u + 3]) + bv.w;
+            }
+          }
           if (EPI == EPI_LSE_PART) {
-            // running (max, sum of 2^(z - max)) of this row over the chunks this warp group sees
-            if (nc + CH > pN) {                          // CTA-uniform: the last, ragged chunk
+            // (ref, sum of 2^(z log2e - ref)) of this row over the chunks this warp group sees.
+            // ref need not be the maximum: it only has to keep the sum inside the fp32 range.  It
+            // stays where it is, from chunk to chunk and from tile to tile (another row's logits
+            // are of the same size as a rule), while a chunk's sum comes out moderate, and moves
+            // to the chunk's maximum otherwise (always for a thread's first chunk, where it is
+            // still -inf).  The common case costs no comparison per element.
+            if (nc + CH > pNt) {                         // CTA-uniform: the last, ragged chunk
 #pragma unroll
               for (int e = 0; e < 32; ++e)
-                if (nc + e >= pN) z[e] = -INFINITY;      // pad columns do not count
+                if (nc + e >= pNt) z[e] = -INFINITY;     // pad columns do not count
             }
-            // four independent chains each, so that the maxima, the ex2 and the sums overlap
-            float m4[4] = {z[0], z[1], z[2], z[3]};
-#pragma unroll
-            for (int e = 4; e < 32; ++e) m4[e & 3] = fmaxf(m4[e & 3], z[e]);
-            const float mn = fmaxf(run_max, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));   // finite: column nc is inside N
+            // four independent chains, so that the ex2 and the sums overlap
             float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int e = 0; e < 32; ++e) s4[e & 3] += ex2_approx(z[e] - mn);
-            run_sum = fmaf(run_sum, ex2_approx(run_max - mn), (s4[0] + s4[1]) + (s4[2] + s4[3]));
-            run_max = mn;
+            for (int e = 0; e < 32; ++e) s4[e & 3] += ex2_approx(fmaf(z[e], kLog2e, -run_max));
+            float cs = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+            // Too large (2^64 or more; the exponent field also catches infinities and NaN, inf - inf
+            // on the pad columns of a thread's first chunk), or too small (below 2^-64) at the
+            // start of a tile: take the reference from this chunk.  A small chunk sum later in a
+            // tile is simply added: the tile's sum so far is at least 2^-64 and dwarfs what a
+            // flush to zero could lose.
+            const uint32_t cs_exp = (__float_as_uint(cs) >> 23) & 0xffu;
+            if (cs_exp >= 127u + 64u || (cs_exp < 127u - 64u && run_sum == 0.f)) {
+              float m4[4] = {z[0], z[1], z[2], z[3]};
+#pragma unroll
+              for (int e = 4; e < 32; ++e) m4[e & 3] = fmaxf(m4[e & 3], z[e]);
+              // finite: column nc is a column of the product (N is padded by less than a chunk)
+              const float mn = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * kLog2e;
+              // the tile's sum so far moves to the new reference, which is higher if there is a sum
+              if (run_sum != 0.f) run_sum *= ex2_approx(run_max - mn);
+              run_max = mn;
+              s4[0] = s4[1] = s4[2] = s4[3] = 0.f;
+#pragma unroll
+              for (int e = 0; e < 32; ++e) s4[e & 3] += ex2_approx(fmaf(z[e], kLog2e, -mn));
+              cs = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+            }
+            run_sum += cs;
           } else {
+            // softmax / rows = 2^(z log2e - (lse log2e + log2 rows))
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
               float o[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) o[e] = ex2_approx(z[8 * u + e] - row_lse) * a.inv_rows;
+              for (int e = 0; e < 8; ++e) o[e] = ex2_approx(fmaf(z[8 * u + e], kLog2e, -row_lse));
               *b16_unit(b16, r, u) = pack8(o);
             }
-            if (nc + CH > pN) {                          // zero the pad columns of the ragged chunk
+            if (nc + CH > pNt) {                         // zero the pad columns of the ragged chunk
 #pragma unroll
               for (int e = 0; e < 32; ++e)
-                if (nc + e >= pN)
+                if (nc + e >= pNt)
                   reinterpret_cast<bf16*>(b16_unit(b16, r, e >> 3))[e & 7] = __float2bfloat16_rn(0.f);
             }
             const int lat = row_label - nc;              // the label's column, if it is in this chunk
@@ -804,8 +869,8 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
               for (int e = 0; e < 32; ++e)
                 if (e == lat) zl = z[e];
               reinterpret_cast<bf16*>(b16_unit(b16, r, lat >> 3))[lat & 7] =
-                  __float2bfloat16_rn((ex2_approx(zl - row_lse) - 1.f) * a.inv_rows);
-              a.label_logit[(long long)g * a.lse_sg + row] = zl * 0.6931471805599453f;
+                  __float2bfloat16_rn(ex2_approx(fmaf(zl, kLog2e, -row_lse)) - a.inv_rows);
+              a.label_logit[(long long)g * a.lse_sg + row] = zl;
             }
           }
         } else {
@@ -837,19 +902,20 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
       }
       if (!ok) break;
       if (EPI == EPI_LSE_PART && row < pM) {
-        // two partials per tile (one per warp group), combined by lse_combine
-        a.lse_part[((long long)g * (2 * p_ntiles) + 2 * at.nt + wg) * pM + row] = make_float2(run_max, run_sum);
+        // one partial per tile and warp group, combined by lse_combine
+        a.lse_part[((long long)g * (NG * p_ntiles) + NG * at.nt + wg) * pM + row] = make_float2(run_max, run_sum);
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {   // the accumulator is free again: tell the CTA that issues the MMAs
-        if (PAIR == 2) mbar_arrive_cluster(map_to_cta(&acc_empty[b], 0)); else mbar_arrive(&acc_empty[b]);
+        if (PAIR == 2) mbar_arrive_cluster<!(EPI == EPI_LSE_PART || EPI == EPI_SOFTMAX_DELTA)>(map_to_cta(&acc_empty[b], 0));
+        else mbar_arrive(&acc_empty[b]);
       }
       ++j;
     }
-  } else if (warp == kAuxWarp) {
+  } else if (ET::kAux && warp == kAuxWarp) {
     // ---------------------------------------------------------------- epilogue input loads
-    if (ET::kAux && lane == 0) {
+    if (lane == 0) {
       int cq = 0, pi = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
@@ -880,7 +946,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         }
       }
     }
-  } else {
+  } else if (warp < kStoreWarp0 + kStoreWarps) {
     // ---------------------------------------------------------------- chunk stores
     if (kStore && lane == 0) {
       const int sj = warp - kStoreWarp0;
@@ -1234,8 +1300,8 @@ TileChoice pick_tile(const GemmArgs<bf16>* a, int n, int epi) {
   return {64, 1};
 }
 
-// Partials per row the EPI_LSE_PART epilogue writes: two per 256-column tile.
-int gemm_tc_lse_parts(int64_t n_store) { return 2 * (int)ceil_div(n_store, 256); }
+// Partials per row the EPI_LSE_PART epilogue writes: one per 256-column tile and warp group.
+int gemm_tc_lse_parts(int64_t n_store) { return (epi_warps(EPI_LSE_PART) / 4) * (int)ceil_div(n_store, 256); }
 
 // Number of k slices gemm_tc will really use when `want` are asked for (slices hold whole
 // 64-deep k blocks, so the count can come out smaller).
@@ -1306,7 +1372,7 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
     const GemmArgs<bf16>& a = ga[i];
     const int n_store = a.N_store > 0 ? a.N_store : a.N;
     TcProblem& p = t.p[i];
-    p.M = a.M; p.N = n_store; p.K = a.K;
+    p.M = a.M; p.N = n_store; p.n_true = a.N; p.K = a.K;
     p.m_tiles = (int)ceil_div(a.M, BM * pair);
     p.n_tiles = (int)ceil_div(n_store, bn);
     p.G = a.G;
@@ -1417,8 +1483,8 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
       if (pair == 2) return launch<0, 1, 256, 4, 1, EPI_LSE_PART, 2>(L, m, t);
       return launch<0, 1, 256, 3, 1, EPI_LSE_PART, 1>(L, m, t);
     case EPI_SOFTMAX_DELTA:
-      if (pair == 2) return launch<0, 1, 256, 4, 6, EPI_SOFTMAX_DELTA, 2>(L, m, t);
-      return launch<0, 1, 256, 3, 6, EPI_SOFTMAX_DELTA, 1>(L, m, t);
+      if (pair == 2) return launch<0, 1, 256, 4, 8, EPI_SOFTMAX_DELTA, 2>(L, m, t);
+      return launch<0, 1, 256, 3, 8, EPI_SOFTMAX_DELTA, 1>(L, m, t);
     case EPI_RELU_MASK:
       if (pair == 2) return launch<0, 0, 256, 6, 4, EPI_RELU_MASK, 2>(L, m, t);
       if (bn == 256) return launch<0, 0, 256, 4, 4, EPI_RELU_MASK, 1>(L, m, t);

@@ -100,8 +100,8 @@ struct GemmArgs {
   const T* mask; int64_t mask_ld, mask_sg;
   bf16* opw;
   float lr;
-  // wide softmax head.  lse_part: [G][2 * ceil(N_store / 256)][M] float2 (two partials per 256-column
-  // tile); lse / label_logit: [G][lse_sg]; labels: labels[g * labels_sg + m].
+  // wide softmax head.  lse_part: [G][gemm_tc_lse_parts(N_store)][M] float2 (a few partials per
+  // 256-column tile); lse / label_logit: [G][lse_sg]; labels: labels[g * labels_sg + m].
   float* lse_part;
   const float* lse; int64_t lse_sg;
   const int32_t* labels; int64_t labels_sg;
