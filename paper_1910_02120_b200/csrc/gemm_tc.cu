@@ -119,7 +119,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = clock64();
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
+    // A try_wait comes back after a fraction of a microsecond whatever its hint says, so a waiting
+    // warp goes round this loop millions of times per second: the abort flag and the clock are
+    // looked at once in 32 rounds, which keeps a round at a few instructions (in the softmax
+    // passes over a very wide output layer, sixteen waiting epilogue warps otherwise issue more
+    // instructions in this loop than in their arithmetic; no measurable difference in time).
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (clock64() - t0 > limit_cycles) {
       *abort_flag = 1;
