@@ -144,6 +144,7 @@ def test_fp32_round_tiny_config():
     ([16, 2500, 6], 5, 4, 1),            # more than one staged column chunk
     ([32] + [64] * 10 + [10], 2, 16, 2), # eleven layers: the bias update takes more than one launch
     ([16, 8, 8, 4], 8, 8, 2),            # one neuron per group
+    ([128, 8192, 10], 2, 640, 2),        # forward product large enough for the 128 x 128 CUDA-core tiles
 ])
 def test_fp32_round_shapes(dims, S, B, K):
     _check_round(_wl("s", dims, S, B, K, "fp32", lr=0.05), FP32_RTOL, 1e-3, FP32_RTOL, True)
@@ -260,7 +261,12 @@ def test_two_rounds_in_a_row_resample():
 # eval
 # ---------------------------------------------------------------------------------------------
 
-@pytest.mark.parametrize("dims,n,B", [([20, 37, 5], 50, 16), ([64, 128, 96, 10], 300, 128)])
+@pytest.mark.parametrize("dims,n,B", [
+    ([20, 37, 5], 50, 16), ([64, 128, 96, 10], 300, 128),
+    # wide enough for the 128 x 128 CUDA-core tiles, ragged in rows, columns and depth: with rows
+    # that take 16-byte loads, and with odd widths that do not
+    ([200, 3304, 3300, 10], 700, 700), ([203, 3301, 3302, 10], 700, 700),
+])
 def test_eval_matches_oracle(dims, n, B):
     import torch
     from oracle import ist_oracle as O
