@@ -175,6 +175,7 @@ class ClockSampler:
         self.gpu = gpu_index
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.p = None
+        self.skip = 0
 
     def start(self):
         try:
@@ -182,6 +183,13 @@ class ClockSampler:
                                        "-lms", "25", "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
+
+    def mark(self):
+        """The timed region starts here: lines written so far belong to the warm-up."""
+        try:
+            self.skip = sum(1 for l in open(self.f.name) if l.strip())
+        except OSError:
+            self.skip = 0
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
@@ -193,7 +201,7 @@ class ClockSampler:
         except Exception:
             self.p.kill()
         self.f.flush()
-        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()][self.skip:]
         os.unlink(self.f.name)
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
@@ -387,13 +395,16 @@ def run_ours(args, w):
         torch.cuda.synchronize(dev)
 
     # ---- device-resident timing ---------------------------------------------------------------
+    # the clock sampler (an nvidia-smi process) needs a few hundred milliseconds before its first
+    # line: it starts before the warm-up rounds, and only the lines written after mark() count
     n_warm = args.warmup if args.quick else max(args.warmup, 3)
+    sampler = ClockSampler(local)
+    sampler.start()
     for i in range(n_warm):
         one_round(i, X_of(dev_in), y_dev)
     ctx.sync_status()
-    sampler = ClockSampler(local)
     barrier()
-    sampler.start()
+    sampler.mark()
     launches0 = ctx.kernel_launches()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
