@@ -288,6 +288,7 @@ struct TcProblem {
   int M, N, K;            // M, N: bounds of the output rows / columns the epilogue touches
   int n_true;             // columns of the product proper (<= N; the rest pads the rows): the softmax passes count only these
   int m_tiles, n_tiles, G;
+  uint32_t m_div, m_sh, n_div, n_sh;   // division by m_tiles / n_tiles as a multiplication, see div_by
   int k_splits, kb_per_split;   // the k range may be cut into slices that run as separate tiles
   int a_gmul, b_gmul;     // 1 if the operand has one slab per group, 0 if all groups share it
   int tile_end;
@@ -333,17 +334,29 @@ struct TcMaps {
 struct TileAt {
   int pi, mt, nt, slab;
 };
+// n / d for 0 <= n < 2^31 with mul = floor(2^(31 + sh) / d) + 1, sh = ceil(log2 d) (set_div): the
+// product over-estimates n / d by less than n / 2^31 / d < 1 / d, so the floor is exact.  Every
+// role of the kernel locates every tile; two hardware divisions per tile were a large share of the
+// instructions of launches with short tiles.
+__device__ __forceinline__ int div_by(int n, uint32_t mul, uint32_t sh) {
+  return (int)(((unsigned long long)(uint32_t)n * mul) >> (31 + sh));
+}
 __device__ __forceinline__ TileAt locate(const TcArgs& a, int tile, int& pi) {
   while (tile >= a.p[pi].tile_end) ++pi;       // tiles are visited in increasing order
   const TcProblem& pr = a.p[pi];
   const int lt = tile - (pi ? a.p[pi - 1].tile_end : 0);
   TileAt t;
   t.pi = pi;
-  t.mt = lt % pr.m_tiles;
-  t.nt = (lt / pr.m_tiles) % pr.n_tiles;
-  t.slab = lt / (pr.m_tiles * pr.n_tiles);
+  const int q = div_by(lt, pr.m_div, pr.m_sh);       // lt / m_tiles
+  t.mt = lt - q * pr.m_tiles;
+  t.slab = div_by(q, pr.n_div, pr.n_sh);             // lt / (m_tiles * n_tiles)
+  t.nt = q - t.slab * pr.n_tiles;
   return t;
 }
+
+// Group and k slice of an output slab; launches without k slices (nearly all) skip the division.
+__device__ __forceinline__ int group_of(const TcProblem& pr, int slab) { return pr.k_splits == 1 ? slab : slab / pr.k_splits; }
+__device__ __forceinline__ int kslice_of(const TcProblem& pr, int slab) { return pr.k_splits == 1 ? 0 : slab % pr.k_splits; }
 
 // Whether tile (mt, nt) of group g has any output inside the group's true extents, and how many
 // 64-deep k blocks its contraction really needs (at least one, so that the accumulator is
@@ -525,11 +538,11 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         const CUtensorMap* tmB = &maps.b[pi];
         const int m0 = at.mt * (BM * PAIR) + rank * BM;     // this CTA's rows of A
         const int n0 = at.nt * BN + rank * BNL;             // this CTA's rows of B
-        const int g = at.slab / pr.k_splits;
+        const int g = group_of(pr, at.slab);
         int kb_limit;
         if (!tile_live<BM * PAIR, BN>(pr, at, g, &kb_limit)) continue;
         const int num_kb = min((pr.K + BK - 1) / BK, kb_limit);
-        const int kb0 = (at.slab % pr.k_splits) * pr.kb_per_split, kb1 = min(num_kb, kb0 + pr.kb_per_split);
+        const int kb0 = kslice_of(pr, at.slab) * pr.kb_per_split, kb1 = min(num_kb, kb0 + pr.kb_per_split);
         const int ga = g * pr.a_gmul, gb = g * pr.b_gmul;
         if (pr.wait_ctr) {
           // A is the output of the problem before this one: wait until every chunk of these rows
@@ -623,14 +636,14 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         const TileAt at = locate(a, tile, pi);
         const TcProblem& pr = a.p[pi];
         int kb_limit;
-        if (!tile_live<BM * PAIR, BN>(pr, at, at.slab / pr.k_splits, &kb_limit)) continue;
+        if (!tile_live<BM * PAIR, BN>(pr, at, group_of(pr, at.slab), &kb_limit)) continue;
         const int b = j & 1;
         ok = mbar_wait(&acc_empty[b], ((j >> 1) & 1) ^ 1, abortp, a.status, 2);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(b * BN);
         const int num_kb = min((pr.K + BK - 1) / BK, kb_limit);
-        const int kb0 = (at.slab % pr.k_splits) * pr.kb_per_split;
+        const int kb0 = kslice_of(pr, at.slab) * pr.kb_per_split;
         const int kb1 = min(num_kb, kb0 + pr.kb_per_split);
         const bool sums = kSums && sums_bias(pr, at);   // the summing warps follow this tile
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -677,12 +690,13 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
     float next_bias[NCH];
     float next_lse = 0.f;
     int next_label = -1;
+    TileAt at_next{};                                 // the tile the last prefetch located: the next one to work on
     auto prefetch_tile_inputs = [&](int tile) {
-      const TileAt at = locate(a, tile, pi_next);
+      const TileAt at = at_next = locate(a, tile, pi_next);
       const TcProblem& pr = a.p[pi_next];
       const int n0 = at.nt * BN;
       if (EPI == EPI_BIAS_RELU || EPI == EPI_BIAS_F32) {
-        const float* bias = pr.bias ? pr.bias + (long long)(at.slab / pr.k_splits) * pr.bias_sg : nullptr;
+        const float* bias = pr.bias ? pr.bias + (long long)group_of(pr, at.slab) * pr.bias_sg : nullptr;
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
           const int n = n0 + c * CH + lane;
@@ -705,10 +719,11 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
     for (int c = 0; c < NCH; ++c) next_bias[c] = 0.f;
     if (unit < total_tiles) prefetch_tile_inputs(unit);
     for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
-      const TileAt at = locate(a, tile, pi);
+      const TileAt at = at_next;                      // located when its inputs were requested
+      pi = at.pi;
       {
         int kb_limit;
-        if (!tile_live<BM * PAIR, BN>(a.p[pi], at, at.slab / a.p[pi].k_splits, &kb_limit)) {
+        if (!tile_live<BM * PAIR, BN>(a.p[pi], at, group_of(a.p[pi], at.slab), &kb_limit)) {
           // the inputs requested for this tile are dropped; ask for the next tile's
           if (tile + n_units < total_tiles) prefetch_tile_inputs(tile + n_units);
           continue;
@@ -929,7 +944,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         const TileAt at = locate(a, tile, pi);
         {
           int kb_limit;
-          if (!tile_live<BM * PAIR, BN>(a.p[pi], at, at.slab / a.p[pi].k_splits, &kb_limit)) continue;
+          if (!tile_live<BM * PAIR, BN>(a.p[pi], at, group_of(a.p[pi], at.slab), &kb_limit)) continue;
         }
         const int pN = a.p[pi].N;
         const int m0 = at.mt * (BM * PAIR) + rank * BM;
@@ -964,13 +979,13 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         const TcProblem& pr = a.p[pi];
         {
           int kb_limit;
-          if (!tile_live<BM * PAIR, BN>(pr, at, at.slab / pr.k_splits, &kb_limit)) {
+          if (!tile_live<BM * PAIR, BN>(pr, at, group_of(pr, at.slab), &kb_limit)) {
             // A skipped tile still counts towards its row block, so that the rows' readers wait for
             // the same total whatever the group's extent (they never read behind the extent).
             if (pr.signal_ctr && sj == 0) {
               const int live = min(NCH, (pr.N - at.nt * BN + CH - 1) / CH);
               if (live > 0)
-                red_release_add(pr.signal_ctr + (long long)(at.slab / pr.k_splits) * pr.m_tiles + at.mt, (unsigned)live);
+                red_release_add(pr.signal_ctr + (long long)group_of(pr, at.slab) * pr.m_tiles + at.mt, (unsigned)live);
             }
             continue;
           }
@@ -1023,7 +1038,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
           // have completed, add them to the row block's count (release: the reader acquires it)
           tma_wait_all();
           fence_proxy_async_all();
-          red_release_add(pr.signal_ctr + (long long)(g / pr.k_splits) * pr.m_tiles + at.mt, stored);
+          red_release_add(pr.signal_ctr + (long long)group_of(pr, g) * pr.m_tiles + at.mt, stored);
         }
       }
       tma_wait_all();                // all stores complete before the CTA exits
@@ -1329,6 +1344,14 @@ bool gemm_tc_update_sums_bias(const GemmArgs<bf16>* a, int n) {
 // Counters a chain of n problems over G groups and up to max_rows output rows needs.
 size_t gemm_tc_chain_counters(int n, int G, int max_rows) { return (size_t)n * G * ceil_div(max_rows, BM); }
 
+// Multiplier and shift of div_by for the divisor d >= 1.
+static void set_div(int d, uint32_t* mul, uint32_t* sh) {
+  uint32_t s = 0;
+  while ((1ull << s) < (unsigned long long)d) ++s;
+  *sh = s;
+  *mul = (uint32_t)((1ull << (31 + s)) / (unsigned long long)d + 1);
+}
+
 bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmChain* chain, const LossReduce* loss,
                    DeviceStatus* st) {
   if (n < 1 || n > kMaxProblems) return false;
@@ -1382,6 +1405,8 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
     p.M = a.M; p.N = n_store; p.n_true = a.N; p.K = a.K;
     p.m_tiles = (int)ceil_div(a.M, BM * pair);
     p.n_tiles = (int)ceil_div(n_store, bn);
+    set_div(p.m_tiles, &p.m_div, &p.m_sh);
+    set_div(p.n_tiles, &p.n_div, &p.n_sh);
     p.G = a.G;
     p.k_splits = 1;
     p.kb_per_split = (int)ceil_div(a.K, BK);

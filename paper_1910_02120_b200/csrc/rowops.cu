@@ -257,13 +257,23 @@ __global__ void __launch_bounds__(1024) lse_combine_kernel(const float2* __restr
   float m = -INFINITY, s = 0.f;
   if (b < B) {
     const float2* p = part + (int64_t)g * parts * B + b;
-#pragma unroll 4
-    for (int i = ty; i < parts; i += 32) {
-      const float2 v = p[(int64_t)i * B];
-      if (v.x > -INFINITY) {                       // an empty partial carries (-inf, 0)
-        const float mn = fmaxf(m, v.x);
-        s = s * exp2f(m - mn) + v.y * exp2f(v.x - mn);
-        m = mn;
+    // eight partials are requested before the first is folded in: a very wide layer has ten
+    // thousand of them per row and only a few dozen blocks to read them
+    constexpr int kAhead = 8;
+    for (int i0 = ty; i0 < parts; i0 += 32 * kAhead) {
+      float2 v[kAhead];
+#pragma unroll
+      for (int u = 0; u < kAhead; ++u) {
+        const int i = i0 + 32 * u;
+        v[u] = i < parts ? p[(int64_t)i * B] : make_float2(-INFINITY, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < kAhead; ++u) {
+        if (v[u].x > -INFINITY) {                  // an empty partial carries (-inf, 0)
+          const float mn = fmaxf(m, v[u].x);
+          s = s * exp2f(m - mn) + v[u].y * exp2f(v[u].x - mn);
+          m = mn;
+        }
       }
     }
   }
