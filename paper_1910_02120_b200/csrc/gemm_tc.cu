@@ -73,16 +73,17 @@ constexpr int CH = 32;                   // epilogue chunk: 32 output columns
 // Warps of a CTA, see the role list above: loader, MMA issuer, the epilogue warps (two groups of
 // four; four groups for the two softmax passes over a very wide output layer, whose epilogues are
 // long chains of dependent instructions and need more warps to hide them), the epilogue input
-// loader, four storers, and two summing warps for weight-update launches on single CTAs.
+// loader, four storers, and two summing warps for weight-update launches (bias gradient).
 constexpr int kSumWarps = 2;
-constexpr bool sums_in_kernel(int epi, int pair) { return epi == 3 /* EPI_SGD */ && pair == 1; }
+constexpr bool sums_in_kernel(int epi, int pair) { return epi == 3 /* EPI_SGD */ && pair == 1; }   // sums from the B stages
+constexpr bool has_sum_warps(int epi) { return epi == 3 /* EPI_SGD */; }
 constexpr int epi_warps(int epi) { return (epi == 5 /* EPI_LSE_PART */ || epi == 6 /* EPI_SOFTMAX_DELTA */) ? 16 : 8; }
 constexpr bool has_aux(int epi) { return epi == 2 /* EPI_RELU_MASK */ || epi == 3; }   // EpiTraits::kAux
 // storers: none where the epilogue stores no chunks (EpiTraits::k32 || k16), two beside sixteen
 // epilogue warps (20 warps leave a thread 96 registers, 22 would leave 80), else four
 constexpr int store_warps(int epi) { return epi == 5 ? 0 : epi == 6 ? 2 : 4; }
 constexpr int threads_for(int epi, int pair) {
-  return (2 + epi_warps(epi) + (has_aux(epi) ? 1 : 0) + store_warps(epi) + (sums_in_kernel(epi, pair) ? kSumWarps : 0)) * 32;
+  return (2 + epi_warps(epi) + (has_aux(epi) ? 1 : 0) + store_warps(epi) + (has_sum_warps(epi) ? kSumWarps : 0)) * 32;
 }
 constexpr long long kWaitLimitCycles = 2000000000ll;   // ~1 s at 2 GHz
 constexpr uint32_t kSuspendHintNs = 20000;             // a waiting thread may sleep this long inside one try_wait
@@ -294,8 +295,13 @@ struct TcProblem {
   int tile_end;
   // true extents of the groups (null: every group fills M / N / K), see GemmArgs
   const int32_t* m_off; const int32_t* n_off; const int32_t* k_off;
-  // weight-update launches: bias[g * bias_upd_sg + n] -= lr * sum_k B[g](n, k) for n < bias_n (null: none)
+  // weight-update launches: bias[g * bias_upd_sg + n] -= lr * sum_k B[g](n, k) for n < bias_n (null: none),
+  // summed from the B stages in shared memory (single CTAs only) ...
   float* bias_upd; long long bias_upd_sg; int bias_n;
+  // ... or the same from B as it lies in memory (bias_mem null: none): dmem[g * dmem_sg + k * dmem_ld + n];
+  // the work is cut into items of 64 columns of one group, items bias_item_end(previous) ..
+  // bias_item_end - 1 of the launch belong to this problem
+  float* bias_mem; const bf16* dmem; long long dmem_ld, dmem_sg; int bias_item_end;
   int head_f32;           // EPI_BIAS_RELU launches only: this problem writes plain fp32 products in
                           // 16-column chunks through the c32 map (a narrow output layer riding on the
                           // hidden layers' launch); 0 = the launch's ordinary epilogue
@@ -313,6 +319,7 @@ struct TcArgs {
   // loss.row_loss[g][0 .. loss_B) for g < loss_G (loss_out null: none)
   LossReduce loss;
   int loss_B, loss_G;
+  int n_bias_items;        // bias items of all problems (see TcProblem::bias_mem)
   float lr;
   DeviceStatus* status;
   // wide softmax head (see GemmArgs); single-problem launches only
@@ -1044,9 +1051,15 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
       tma_wait_all();                // all stores complete before the CTA exits
     }
   }
-  if (kSums && warp >= kStoreWarp0 + kStoreWarps) {
+  if (has_sum_warps(EPI) && warp >= kStoreWarp0 + kStoreWarps) {
     // ---------------------------------------------------------------- bias gradient (and loss means)
-    // Summing warp sw owns the 64-column box sw of the B tile (MN-major: row k of a box holds 64
+    // Two ways, chosen by the host per launch.  From memory (bias_mem): while the deltas of a step
+    // are small enough to be still in L2, the summing warps of all CTAs share out (group, 64
+    // columns) items and read them with plain loads, sixteen rows in flight per lane, at their own
+    // pace beside the tiles: no barrier of the pipeline knows of them.  From shared memory
+    // (bias_upd, single CTAs): deltas that no longer fit in L2 would come from DRAM a second time,
+    // so there the warps read them out of the B stages as they pass:
+    // summing warp sw owns the 64-column box sw of the B tile (MN-major: row k of a box holds 64
     // consecutive columns, 128 bytes, 16-byte units swizzled by k % 8); lane l adds up columns
     // 8 (l % 8) .. + 7 over the rows k = l / 8 (mod 4), and the four lanes of a column combine
     // their sums at the end of the tile.  Only the first tile row carries a bias update
@@ -1067,11 +1080,39 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, const __grid_constant__ TcAr
         if (lane == 0) a.loss.loss_out[(long long)g * a.loss.out_stride + a.loss.k] = acc / (float)a.loss_B;
       }
     }
+    if (a.n_bias_items > 0) {
+      const int n_workers = (int)gridDim.x * kSumWarps;
+      int pj = 0;
+      for (int item = (int)blockIdx.x * kSumWarps + sw; item < a.n_bias_items; item += n_workers) {
+        while (item >= a.p[pj].bias_item_end) ++pj;
+        const TcProblem& pr = a.p[pj];
+        const int li = item - (pj ? a.p[pj - 1].bias_item_end : 0);
+        const int blocks = (pr.bias_n + 63) / 64;            // column blocks of a group
+        const int g = li / blocks, c0 = (li - g * blocks) * 64 + 2 * lane;   // this lane's two columns
+        if (c0 >= pr.bias_n) continue;                       // rows are padded to an even length
+        const uint32_t* dp = reinterpret_cast<const uint32_t*>(pr.dmem + (long long)g * pr.dmem_sg + c0);
+        const long long ld2 = pr.dmem_ld / 2;
+        float acc0 = 0.f, acc1 = 0.f;
+        for (int r0 = 0; r0 < pr.K; r0 += 16) {              // the contraction of a weight update runs over the batch
+          uint32_t v[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = r0 + i < pr.K ? __ldg(dp + (long long)(r0 + i) * ld2) : 0u;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {                     // rows in ascending order: a fixed sum
+            acc0 += __uint_as_float(v[i] << 16);
+            acc1 += __uint_as_float(v[i] & 0xffff0000u);
+          }
+        }
+        float* bp = pr.bias_mem + (long long)g * pr.bias_upd_sg + c0;
+        bp[0] -= a.lr * acc0;
+        if (c0 + 1 < pr.bias_n) bp[1] -= a.lr * acc1;
+      }
+    }
     constexpr int kBoxes = BNL / 64;
     static_assert(!kSums || kBoxes <= kSumWarps, "one summing warp per 64-column box");
     int it = 0, pi = 0, sit = 0;
     bool ok = true;
-    for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
+    for (int tile = unit; kSums && tile < total_tiles && ok; tile += n_units) {
       const TileAt at = locate(a, tile, pi);
       const TcProblem& pr = a.p[pi];
       int kb_limit;
@@ -1391,13 +1432,13 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
   t.labels = a0.labels; t.labels_sg = a0.labels_sg;
   t.label_logit = a0.label_logit;
   t.inv_rows = a0.inv_rows;
-  if (loss && (epi != EPI_SGD || pair != 1)) return false;
+  if (loss && epi != EPI_SGD) return false;
   if (loss) {
     t.loss = *loss;
     t.loss_B = a0.K;          // the contraction of a weight update runs over the batch
     t.loss_G = a0.G;
   }
-  int64_t tiles = 0;
+  int64_t tiles = 0, bias_items = 0;
   for (int i = 0; i < n; ++i) {
     const GemmArgs<bf16>& a = ga[i];
     const int n_store = a.N_store > 0 ? a.N_store : a.N;
@@ -1422,8 +1463,19 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
     p.b_gmul = (a.G > 1 && a.b_sg != 0) ? 1 : 0;
     p.bias = a.bias; p.bias_sg = a.bias_sg;
     p.m_off = a.m_off; p.n_off = a.n_off; p.k_off = a.k_off;
-    if (a.bias_upd && (epi != EPI_SGD || pair != 1)) return false;   // see gemm_tc_update_sums_bias
-    p.bias_upd = a.bias_upd; p.bias_upd_sg = a.bias_upd_sg; p.bias_n = a.bias_n;
+    if (a.bias_upd && epi != EPI_SGD) return false;
+    p.bias_upd_sg = a.bias_upd_sg; p.bias_n = a.bias_n;
+    p.bias_item_end = bias_items;
+    if (a.bias_upd && a.bias_upd_from_memory) {
+      if (!b_mn || a.b_sk % 2 != 0 || a.b_sg % 2 != 0 || reinterpret_cast<uintptr_t>(a.B) % 4 != 0) return false;
+      p.bias_mem = a.bias_upd; p.dmem = a.B; p.dmem_ld = a.b_sk; p.dmem_sg = a.G > 1 ? a.b_sg : 0;
+      bias_items += (int64_t)a.G * ceil_div(a.bias_n, 64);
+      if (bias_items > 0x7fffffffll) return false;
+      p.bias_item_end = (int)bias_items;
+    } else if (a.bias_upd) {
+      if (pair != 1) return false;   // sums from the B stages: single CTAs only, see gemm_tc_update_sums_bias
+      p.bias_upd = a.bias_upd;
+    }
     if (a.k_off && p.k_splits > 1) return false;
     tiles += (int64_t)p.m_tiles * p.n_tiles * p.G * p.k_splits;
     if (tiles > 0x7fffffffll) return false;
@@ -1476,6 +1528,7 @@ bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* ga, int n, const GemmC
     }
   }
   t.total_tiles = (int)tiles;
+  t.n_bias_items = (int)bias_items;
   if (chain) {
     // Problem i + 1 reads problem i's output rows: same groups, same rows, hence the same tile rows.
     // Every CTA of a unit stores ceil(N / 32) chunks per (group, tile row) and launch; the running

@@ -684,21 +684,22 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       upd.push_back(g);
     }
     // Biases are not read by the backward pass, so their update may come before or after the
-    // weight updates.  While the deltas it sums are small enough to be still in L2, the bias
-    // kernel runs first and costs next to nothing.  Deltas beyond that size (a very wide output
-    // layer) would be read from memory a second time: there the weight-update launch, when it
-    // runs on single CTAs, sums the deltas it streams anyway (its B operand), updates the biases
-    // itself and reduces the step's mean losses; what is left for the bias kernel is a sparse
-    // first layer's bias.  Otherwise the bias kernel runs last.
+    // weight updates.  With bf16 operands the weight-update launch does it on the side, in two
+    // warps per CTA that sum the deltas and also reduce the step's mean losses: from memory while
+    // the deltas of a step are small enough to be still in L2, out of the operand stages it
+    // streams anyway when they are not (a very wide output layer; single-CTA launches only).
+    // What is left for the bias kernel is a sparse first layer's bias, launches that can do
+    // neither, and the fp32 path, where it runs first if the deltas fit in L2 and last otherwise.
     const bool sparse_first = X->kind == IST_X_CSR && t > 1;
     size_t delta_bytes = 0;
     for (int l = 1; l <= t; ++l) delta_bytes += (size_t)S * B * c->ld[l] * sizeof(T);
     const bool bias_first = delta_bytes <= kL2ResidentBytes;
-    const bool bias_in_gemm = !bias_first && update_sums_bias(upd);
+    const bool bias_in_gemm = bf && (bias_first || update_sums_bias(upd));
     if (bias_in_gemm) {
       for (auto& g : upd) {
-        const int l = (int)(&g - upd.data());   // upd[i] is layer t - i
-        g.bias_upd = bias_of(t - l); g.bias_upd_sg = c->ld[t - l]; g.bias_n = (int)c->np[t - l];
+        const int l = t - (int)(&g - upd.data());   // upd[i] is layer t - i
+        g.bias_upd = bias_of(l); g.bias_upd_sg = c->ld[l]; g.bias_n = (int)c->np[l];
+        g.bias_upd_from_memory = bias_first ? 1 : 0;
       }
       if (sparse_first) update_biases(1, 1, false);
     } else if (bias_first) {

@@ -92,7 +92,9 @@ struct GemmArgs {
   // EPI_SGD on the tensor-core path, launches on single CTAs only (gemm_tc_update_sums_bias): the
   // launch also updates the layer's bias from the B operand (the deltas) it streams anyway:
   // bias_upd[g * bias_upd_sg + n] -= lr * sum_k B[g](n, k), n < bias_n.
-  float* bias_upd; int64_t bias_upd_sg; int bias_n;
+  // bias_upd_from_memory: the deltas are read from memory (any launch shape; meant for deltas that are
+  // still in L2) instead of from the operand stages.
+  float* bias_upd; int64_t bias_upd_sg; int bias_n; int bias_upd_from_memory;
   int epi;
   const float* bias; int64_t bias_sg;
   T* out; int64_t out_ld, out_sg;
@@ -124,8 +126,7 @@ struct GemmChain {
   size_t stride;
   unsigned* totals;
 };
-// loss (weight-update launches on single CTAs only, may be null): the step's mean losses are
-// reduced by the launch.
+// loss (weight-update launches only, may be null): the step's mean losses are reduced by the launch.
 struct LossReduce;
 bool gemm_tc_batch(const Launch& L, const GemmArgs<bf16>* a, int n, const GemmChain* chain, const LossReduce* loss,
                    DeviceStatus* st);
