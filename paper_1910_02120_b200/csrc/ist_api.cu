@@ -685,21 +685,24 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
     }
     // Biases are not read by the backward pass, so their update may come before or after the
     // weight updates.  With bf16 operands the weight-update launch does it on the side, in two
-    // warps per CTA that sum the deltas and also reduce the step's mean losses: from memory while
-    // the deltas of a step are small enough to be still in L2, out of the operand stages it
-    // streams anyway when they are not (a very wide output layer; single-CTA launches only).
-    // What is left for the bias kernel is a sparse first layer's bias, launches that can do
-    // neither, and the fp32 path, where it runs first if the deltas fit in L2 and last otherwise.
+    // warps per CTA that sum the deltas and also reduce the step's mean losses: out of the operand
+    // stages it streams anyway when the deltas of a step are too large to be still in L2 and the
+    // launch runs on single CTAs (a very wide output layer), from memory otherwise (from L2 as a
+    // rule; deltas beyond its size come from DRAM a second time there, as they would for the bias
+    // kernel, but in the shadow of the update).  What is left for the bias kernel is a sparse
+    // first layer's bias and the fp32 path, where it runs first if the deltas fit in L2 and last
+    // otherwise.
     const bool sparse_first = X->kind == IST_X_CSR && t > 1;
     size_t delta_bytes = 0;
     for (int l = 1; l <= t; ++l) delta_bytes += (size_t)S * B * c->ld[l] * sizeof(T);
     const bool bias_first = delta_bytes <= kL2ResidentBytes;
-    const bool bias_in_gemm = bf && (bias_first || update_sums_bias(upd));
+    const bool bias_in_gemm = bf;
+    const bool from_stages = bias_in_gemm && !bias_first && update_sums_bias(upd);
     if (bias_in_gemm) {
       for (auto& g : upd) {
         const int l = t - (int)(&g - upd.data());   // upd[i] is layer t - i
         g.bias_upd = bias_of(l); g.bias_upd_sg = c->ld[l]; g.bias_n = (int)c->np[l];
-        g.bias_upd_from_memory = bias_first ? 1 : 0;
+        g.bias_upd_from_memory = from_stages ? 0 : 1;
       }
       if (sparse_first) update_biases(1, 1, false);
     } else if (bias_first) {
