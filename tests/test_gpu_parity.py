@@ -166,7 +166,8 @@ def test_fp32_round_shapes(dims, S, B, K):
     ([64, 256, 128, 10], 2, 700, 2, "normal"),             # batch larger than 512
     ([16, 8, 8, 4], 8, 8, 2, "normal"),                    # one neuron per group
     ([64, 256, 8192], 2, 64, 2, "normal"),                 # widest output layer that still stores its logits
-    ([64, 256, 70001], 2, 256, 2, "normal"),               # deltas beyond L2 size: the update launch sums them for the biases
+    ([64, 256, 70001], 2, 256, 2, "normal"),               # deltas beyond L2 size, single CTAs: the update launch sums them out of its operand stages
+    ([256, 65536, 10], 8, 512, 2, "normal"),               # deltas beyond L2 size on CTA pairs: summed from memory beside the tiles
 ])
 def test_bf16_round_shapes(dims, S, B, K, x_dist):
     _check_round(_wl("b", dims, S, B, K, "bf16", x_dist=x_dist), BF16_W_RTOL, BF16_DW_RTOL,
