@@ -288,6 +288,20 @@ def gradients(Ws, bs, X, y, dtype=np.float64):
     return loss, dW, db
 
 
+def input_gradient(Ws, bs, X, y, dtype=np.float64):
+    """d(loss)/dX of one minibatch at the current parameters: delta_1 W_1^T, where delta_1 is the
+    gradient with respect to the first layer's pre-activations (back-propagated as in
+    `gradients`).  Sec. 2.2, "IST for other architectures": when only the fully connected part of
+    a network is partitioned, whatever produces its input (a convolutional trunk that every site
+    holds whole) is trained from this gradient.  Dense X only."""
+    t = len(Ws)
+    z, a = forward(Ws, bs, X, dtype)
+    _, delta = softmax_xent(z[t - 1], np.asarray(y, dtype=np.int64))
+    for l in range(t, 1, -1):
+        delta = (delta @ Ws[l - 1].T) * (z[l - 2] > 0)
+    return delta @ Ws[0].T
+
+
 # ----------------------------------------------------------------------------
 # Sec. 2.2 "Correcting Distributional Shift": every hidden neuron's input is
 # standardised with the mean and standard deviation over the minibatch before
@@ -462,6 +476,20 @@ class IstOracle:
                 xb, yb = self._batch(X, y, s, k)
                 losses[s, k] = sgd_step(Ws, bs, xb, yb, lr, self.dtype, self.norm_eps)
         return losses
+
+    def local_steps_dx(self, X, y, lr: float, K: int):
+        """local_steps that also returns dX[s][k] = d(loss of step k)/d(batch of step k), taken at
+        the parameters the step starts from (before its update).  Plain path, dense X."""
+        assert self.norm_eps is None and not isinstance(X, tuple)
+        losses = np.zeros((self.S, K), dtype=np.float64)
+        dX = np.zeros(np.asarray(X).shape, dtype=self.dtype)
+        for s in range(self.S):
+            Ws, bs = self.subnets[s]
+            for k in range(K):
+                xb, yb = self._batch(X, y, s, k)
+                dX[s, k] = input_gradient(Ws, bs, xb, yb, self.dtype)
+                losses[s, k] = sgd_step(Ws, bs, xb, yb, lr, self.dtype, None)
+        return losses, dX
 
     def reassemble(self):
         reassemble(self.W, self.b, self.parts, self.subnets)

@@ -247,6 +247,72 @@ def test_finite_difference_gradients():
                 assert abs(fd - g[i]) <= 1e-6 * max(1.0, abs(g[i])) + 1e-9
 
 
+@pytest.mark.parametrize("dims", [[7, 5], [6, 9, 4], [5, 8, 7, 3]])
+def test_input_gradient_matches_torch_autograd_and_central_differences(dims):
+    # Sec. 2.2 "IST for other architectures": what a trunk in front of the partitioned layers is
+    # trained from.  Pinned twice: against autograd of the same network in torch, and against
+    # central differences of the oracle's own loss in every input entry.
+    W, b, X, y = _tiny(dims, 1, 6, 1, seed=11)
+    Ws = [w.astype(np.float64) for w in W]
+    bs = [v.astype(np.float64) for v in b]
+    x, yy = X[0, 0].astype(np.float64), y[0, 0]
+    dx = O.input_gradient(Ws, bs, x, yy)
+    assert dx.shape == x.shape
+    tx = torch.tensor(x, requires_grad=True)
+    tl = _torch_loss([torch.tensor(w) for w in Ws], [torch.tensor(v) for v in bs], tx,
+                     torch.tensor(yy, dtype=torch.long))
+    tl.backward()
+    np.testing.assert_allclose(dx, tx.grad.numpy(), rtol=1e-10, atol=1e-13)
+
+    def f(xx):
+        z, _ = O.forward(Ws, bs, xx)
+        return O.softmax_xent(z[-1], yy.astype(np.int64))[0]
+
+    z0, _ = O.forward(Ws, bs, x)
+    if len(Ws) > 1:
+        assert min(np.abs(zz).min() for zz in z0[:-1]) > 1e-4      # away from ReLU kinks
+    h = 1e-6
+    for i in range(x.shape[0]):
+        for j in range(x.shape[1]):
+            xp, xm = x.copy(), x.copy()
+            xp[i, j] += h
+            xm[i, j] -= h
+            fd = (f(xp) - f(xm)) / (2 * h)
+            assert abs(fd - dx[i, j]) <= 1e-6 * max(1.0, abs(dx[i, j])) + 1e-9
+
+
+def test_local_steps_dx_is_taken_before_each_update():
+    # dX of step k is the input gradient at the parameters step k starts from; the losses and the
+    # trained slices are those of local_steps
+    dims, S, B, K, lr = [6, 12, 8, 4], 2, 5, 3, 0.05
+    W, b, X, y = _tiny(dims, S, B, K, seed=4)
+    o = O.IstOracle(dims, S)
+    o.bind_weights(W, b)
+    o.partition(9)
+    ref = O.IstOracle(dims, S)
+    ref.bind_weights(W, b)
+    ref.partition(9)
+    losses, dX = o.local_steps_dx(X, y, lr, K)
+    assert dX.shape == X.shape
+    for s in range(S):
+        Ws, bs = ref.subnets[s]
+        for k in range(K):
+            xb, yb = ref._batch(X, y, s, k)
+            np.testing.assert_array_equal(dX[s, k], O.input_gradient(Ws, bs, xb, yb))
+            O.sgd_step(Ws, bs, xb, yb, lr)
+    np.testing.assert_array_equal(losses, O.IstOracle.local_steps(_fresh(dims, S, W, b, 9), X, y, lr, K))
+    for s in range(S):
+        for l in range(len(W)):
+            np.testing.assert_array_equal(o.subnets[s][0][l], ref.subnets[s][0][l])
+
+
+def _fresh(dims, S, W, b, seed):
+    o = O.IstOracle(dims, S)
+    o.bind_weights(W, b)
+    o.partition(seed)
+    return o
+
+
 def test_S1_round_is_plain_sgd():
     # xi = 1 in the paper's compression operator: the mask is the identity and IST is SGD.
     dims, B, K, lr = [6, 10, 8, 4], 7, 5, 0.05
