@@ -181,6 +181,22 @@ ist_status ist_local_steps(ist_ctx* ctx, const ist_input* X, const int32_t* y_de
                            float* loss_out_dev);
 
 /*
+ * Sec. 2.2, "IST for other architectures": when only the fully connected part of a network is
+ * partitioned, the part in front of it (a convolutional trunk, which every site holds whole and
+ * trains by local SGD) needs the gradient of each subnet's loss with respect to that subnet's
+ * inputs.  Same as ist_local_steps, and in addition
+ * dx_out_dev (device, fp32, not NULL): rows addressed exactly like the rows of X (row r of X ->
+ * row r of dx_out_dev, N_0 floats each, so the buffer spans as many rows as X does); the row of
+ * subnet s, step k, sample b receives d(loss[s][k]) / d(that input row) = delta_1 W_1^T on the
+ * subnet's slice, taken at the weights step k starts from.  Rows of X that no step reads are not
+ * written.  Dense inputs only (IST_ERR_UNSUPPORTED for CSR); on the bf16 path N_0 must be a
+ * multiple of 4.  With K > 1 the later steps' gradients belong to inputs the trunk produced
+ * before its own update: the usual call has K = 1.
+ */
+ist_status ist_local_steps_dx(ist_ctx* ctx, const ist_input* X, const int32_t* y_dev, float lr, int K,
+                              float* loss_out_dev, float* dx_out_dev);
+
+/*
  * Training the S subnets at several sites (Sec. 2.1 "Distributing Subnets": every subnet goes to
  * its own compute node; Sec. 2.3: only the slices travel).  A context may own only subnets
  * first .. first + count - 1: ist_partition then draws the whole partition (it is cheap and every

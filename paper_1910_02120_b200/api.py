@@ -26,7 +26,7 @@ EXPORTS = [
     "ist_kernel_launches", "ist_last_error", "ist_destroy", "ist_profile", "ist_profile_read",
     "ist_partition_layer_static", "ist_norm_workspace_bytes", "ist_enable_normalization", "ist_calibrate",
     "ist_set_subnet_range", "ist_packed_layer", "ist_workspace_bytes2", "ist_create2",
-    "ist_selftest_wait_expiry", "ist_subnet_slice_shape", "ist_static_partition_status",
+    "ist_selftest_wait_expiry", "ist_subnet_slice_shape", "ist_static_partition_status", "ist_local_steps_dx",
 ]
 IST_PART_BALANCED, IST_PART_IID = 0, 1
 IST_STATIC_MAX_NEURONS, IST_STATIC_MAX_SUBNETS = 65536, 64
@@ -84,6 +84,8 @@ def _load() -> ctypes.CDLL:
     lib.ist_static_partition_status.argtypes = [vp]
     lib.ist_local_steps.restype = ctypes.c_int32
     lib.ist_local_steps.argtypes = [vp, ctypes.POINTER(IstInput), vp, ctypes.c_float, i32, vp]
+    lib.ist_local_steps_dx.restype = ctypes.c_int32
+    lib.ist_local_steps_dx.argtypes = [vp, ctypes.POINTER(IstInput), vp, ctypes.c_float, i32, vp, vp]
     lib.ist_reassemble.restype = ctypes.c_int32
     lib.ist_reassemble.argtypes = [vp]
     lib.ist_eval.restype = ctypes.c_int32
@@ -277,8 +279,11 @@ class Ist:
 
     def local_steps(self, X, y: torch.Tensor, lr: float, K: int, batch: int,
                     stride_subnet: Optional[int] = None, stride_step: Optional[int] = None,
-                    loss_out: Optional[torch.Tensor] = None, want_loss: bool = True):
-        """X rows ordered [S][K][batch] by default (stride_subnet = K*batch, stride_step = batch)."""
+                    loss_out: Optional[torch.Tensor] = None, want_loss: bool = True,
+                    dx_out: Optional[torch.Tensor] = None):
+        """X rows ordered [S][K][batch] by default (stride_subnet = K*batch, stride_step = batch).
+        dx_out: fp32 [rows of X][N_0], receives the loss gradient with respect to every input row
+        (ist_local_steps_dx)."""
         if stride_subnet is None:
             stride_subnet = K * batch
         if stride_step is None:
@@ -288,8 +293,13 @@ class Ist:
         n_sub = getattr(self, "sub_count", self.S)
         if loss_out is None and want_loss:
             loss_out = torch.empty(n_sub * K, dtype=torch.float32, device=self.device)
-        _check(self.handle, lib.ist_local_steps(self.handle, ctypes.byref(inp), y.data_ptr(),
-                                                ctypes.c_float(lr), K, _ptr(loss_out)))
+        if dx_out is not None:
+            assert dx_out.is_cuda and dx_out.dtype == torch.float32 and dx_out.is_contiguous()
+            _check(self.handle, lib.ist_local_steps_dx(self.handle, ctypes.byref(inp), y.data_ptr(),
+                                                       ctypes.c_float(lr), K, _ptr(loss_out), dx_out.data_ptr()))
+        else:
+            _check(self.handle, lib.ist_local_steps(self.handle, ctypes.byref(inp), y.data_ptr(),
+                                                    ctypes.c_float(lr), K, _ptr(loss_out)))
         return loss_out.view(n_sub, K) if loss_out is not None else None
 
     def reassemble(self):

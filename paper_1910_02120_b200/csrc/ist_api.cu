@@ -435,12 +435,21 @@ void small_softmax(const Launch& L, const float* part, int ks, int64_t ld, int G
                    float* row_loss, DeviceStatus* st) {
   softmax_xent_small<bf16>(L, part, ks, ld, G, B, Nt, bias, bias_sg, y, y_sg, delta, ld_d, sg_d, row_loss, st);
 }
+// A product written as plain fp32: on the tensor-core path the fp32 epilogue without a bias, on
+// the CUDA-core path (operands and output of the same type) a plain store.
+void set_plain_fp32_output(GemmArgs<bf16>& g, float* out, int64_t ld, int64_t sg) {
+  g.epi = EPI_BIAS_F32; g.bias = nullptr; g.outf = out; g.outf_ld = ld; g.outf_sg = sg;
+}
+void set_plain_fp32_output(GemmArgs<float>& g, float* out, int64_t ld, int64_t sg) {
+  g.epi = EPI_STORE; g.out = out; g.out_ld = ld; g.out_sg = sg;
+}
 // Working sets up to this size are taken to survive in the 126 MB L2 between two kernels.
 constexpr size_t kL2ResidentBytes = 64u << 20;
 // One call of ist_local_steps in operand type T.
+// dx_out (may be null): fp32 rows addressed like the rows of X; row r receives d(loss)/d(row r).
 template <typename T>
 ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, float lr, int K,
-                           float* loss_out) {
+                           float* loss_out, float* dx_out) {
   // S here is the number of subnets this context trains: slabs s0 .. s0 + S - 1 of the packed
   // weights; activations, deltas and the other scratch buffers use their first S slabs.
   const int t = c->t, S = c->sub_count, s0 = c->sub_first, B = X->batch;
@@ -667,6 +676,22 @@ ist_status run_local_steps(ist_ctx* c, const ist_input* X, const int32_t* y, flo
       }
     }
     if (!flush_dx()) return fail(c, IST_ERR_UNSUPPORTED, "delta GEMMs cannot be launched");
+    if (dx_out) {
+      // Sec. 2.2, "IST for other architectures": the gradient with respect to the step's inputs,
+      // delta_1 W_1^T on every subnet's slice, taken like all gradients at the weights the step
+      // started from (the update below has not touched them yet).  This is what a trunk in front
+      // of the partitioned layers (held whole at every site) is trained from.
+      Scope sc(c, IST_K_DX);
+      GemmArgs<T> g{};
+      g.M = B; g.N = (int)c->N[0]; g.K = (int)c->np[1]; g.G = S;
+      g.N_store = (int)c->N[0];
+      g.A = delta(1); g.a_sm = c->ld[1]; g.a_sk = 1; g.a_sg = Bm * c->ld[1];
+      g.B = weights(1); g.b_sn = c->ld[1]; g.b_sk = 1; g.b_sg = c->slice_elems(1);
+      g.k_off = t > 1 ? off_of(1) : nullptr;
+      float* out = dx_out + row0 * c->N[0];
+      set_plain_fp32_output(g, out, c->N[0], X->stride_subnet * c->N[0]);
+      if (!gemm(c, g)) return fail(c, IST_ERR_UNSUPPORTED, "input-gradient GEMM cannot be launched (N_0 must be a multiple of 4)");
+    }
     // the weight updates of the dense layers do not depend on one another: tiles of one launch
     std::vector<GemmArgs<T>> upd;
     for (int l = t; l >= 1; --l) {
@@ -907,8 +932,24 @@ extern "C" ist_status ist_local_steps(ist_ctx* c, const ist_input* X, const int3
   if (!(lr == lr)) return fail(c, IST_ERR_ARG, "lr is NaN");
   ist_status s = check_input(c, X, y_dev, true);
   if (s != IST_OK) return s;
-  if (c->precision == IST_BF16) return run_local_steps<bf16>(c, X, y_dev, lr, K, loss_out_dev);
-  return run_local_steps<float>(c, X, y_dev, lr, K, loss_out_dev);
+  if (c->precision == IST_BF16) return run_local_steps<bf16>(c, X, y_dev, lr, K, loss_out_dev, nullptr);
+  return run_local_steps<float>(c, X, y_dev, lr, K, loss_out_dev, nullptr);
+}
+
+extern "C" ist_status ist_local_steps_dx(ist_ctx* c, const ist_input* X, const int32_t* y_dev, float lr,
+                                         int K, float* loss_out_dev, float* dx_out_dev) {
+  if (!c) return IST_ERR_ARG;
+  if (c->state != ST_PARTITIONED) return fail(c, IST_ERR_STATE, "ist_local_steps_dx needs a partition in place");
+  if (K < 1) return fail(c, IST_ERR_ARG, "K must be >= 1");
+  if (!(lr == lr)) return fail(c, IST_ERR_ARG, "lr is NaN");
+  if (!dx_out_dev) return fail(c, IST_ERR_ARG, "dx_out_dev must not be null");
+  ist_status s = check_input(c, X, y_dev, true);
+  if (s != IST_OK) return s;
+  if (X->kind == IST_X_CSR) return fail(c, IST_ERR_UNSUPPORTED, "the input gradient is defined for dense inputs only");
+  if (c->precision == IST_BF16 && c->N[0] % 4 != 0)
+    return fail(c, IST_ERR_UNSUPPORTED, "the input gradient on the bf16 path needs N_0 to be a multiple of 4");
+  if (c->precision == IST_BF16) return run_local_steps<bf16>(c, X, y_dev, lr, K, loss_out_dev, dx_out_dev);
+  return run_local_steps<float>(c, X, y_dev, lr, K, loss_out_dev, dx_out_dev);
 }
 
 extern "C" ist_status ist_set_subnet_range(ist_ctx* c, int first, int count) {
